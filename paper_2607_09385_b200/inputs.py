@@ -1,0 +1,208 @@
+"""Seeded synthetic inputs for the block-sparse fused attention path.
+
+This module serves both the CUDA path's callers (tests, bench) and the CPU oracle's
+callers.  It holds no attention arithmetic: only the workload table, a counter-based
+random generator and the block-bitmap draw.  Everything is produced on the host as
+numpy arrays so that both sides consume identical bytes.
+
+Generator (fixed so results are reproducible across machines and thread counts):
+element with flat index ``e`` of stream ``t`` draws
+
+    x  = splitmix64(seed ^ (t << 60) ^ e),  y = splitmix64(x)
+    u1 = ((x >> 11) + 1) * 2**-53           in (0, 1]
+    u2 = (y >> 11) * 2**-53                 in [0, 1)
+    z  = sqrt(-2 ln u1) * cos(2 pi u2)      standard normal (Box-Muller, fp64)
+
+and the stored value is ``bf16(float32(sigma * s_h * z))`` with round-to-nearest-even
+at both narrowings.  Streams: Q=1, K=2, V=3, per-head query scale=4, bitmap=5.
+
+The workloads follow the paper's evaluation style (random tensors of model-shaped
+attention problems, Sec. "Attention Benchmark"); no dataset is involved.
+"""
+from __future__ import annotations
+
+import dataclasses
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+MASK_CAUSAL = 1
+MASK_WINDOW = 2
+MASK_BITMAP = 4
+
+STREAM_Q, STREAM_K, STREAM_V, STREAM_HEAD_SCALE, STREAM_BITMAP = 1, 2, 3, 4, 5
+DEFAULT_SEED = 0x5EED
+
+_U64 = np.uint64
+_CHUNK = 1 << 22
+
+
+def splitmix64(x: np.ndarray) -> np.ndarray:
+    """One splitmix64 output step on an array of uint64 states (wrapping arithmetic)."""
+    with np.errstate(over="ignore"):
+        z = x + _U64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> _U64(30))) * _U64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> _U64(27))) * _U64(0x94D049BB133111EB)
+        return z ^ (z >> _U64(31))
+
+
+def _uniform_pair(seed: int, stream: int, e: np.ndarray):
+    key = _U64((seed ^ (stream << 60)) & 0xFFFFFFFFFFFFFFFF)
+    x = splitmix64(key ^ e)
+    y = splitmix64(x)
+    u1 = ((x >> _U64(11)).astype(np.float64) + 1.0) * 2.0 ** -53
+    u2 = (y >> _U64(11)).astype(np.float64) * 2.0 ** -53
+    return u1, u2
+
+
+def uniform(seed: int, stream: int, e: np.ndarray) -> np.ndarray:
+    """u1 of the recipe, in (0, 1], for element indices ``e`` of ``stream``."""
+    return _uniform_pair(seed, stream, np.asarray(e, dtype=np.uint64))[0]
+
+
+def normal(seed: int, stream: int, e: np.ndarray) -> np.ndarray:
+    """Standard normal draws (fp64) for element indices ``e`` of ``stream``."""
+    u1, u2 = _uniform_pair(seed, stream, np.asarray(e, dtype=np.uint64))
+    return np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (nearest even); returns the 16-bit patterns."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bfloat16 bit patterns exactly to float64."""
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def normal_bf16(seed: int, stream: int, shape, sigma: float = 1.0,
+                row_scale: np.ndarray | None = None, threads: int = 8) -> np.ndarray:
+    """bf16 bit patterns (uint16) of ``sigma * row_scale * N(0,1)`` with the given shape.
+
+    ``row_scale`` (optional, fp64) has one entry per index of ``shape[:2]`` flattened
+    (batch*heads) and multiplies every element of that head.
+    """
+    n = int(np.prod(shape))
+    out = np.empty(n, dtype=np.uint16)
+    per_head = int(np.prod(shape[2:])) if len(shape) > 2 else 1
+
+    def work(lo: int) -> None:
+        hi = min(lo + _CHUNK, n)
+        e = np.arange(lo, hi, dtype=np.uint64)
+        z = normal(seed, stream, e) * sigma
+        if row_scale is not None:
+            z *= row_scale[(e // _U64(per_head)).astype(np.int64)]
+        out[lo:hi] = f32_to_bf16_bits(z.astype(np.float32))
+
+    starts = range(0, n, _CHUNK)
+    if threads > 1 and n > _CHUNK:
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(work, starts))
+    else:
+        for lo in starts:
+            work(lo)
+    return out.reshape(shape)
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    """One attention problem: shapes, mask descriptor and value recipe."""
+    name: str
+    batch: int
+    heads_q: int
+    heads_kv: int
+    seq: int
+    head_dim: int
+    block: int
+    flags: int
+    window: int = 0
+    keep_prob: float = 0.0        # bitmap: Bernoulli keep probability of non-forced blocks
+    sigma: float = 1.0            # standard deviation of Q, K, V entries
+    head_query_scale: bool = False  # Q of head h multiplied by s_h ~ U[0.5, 2]
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / float(np.sqrt(self.head_dim))
+
+    @property
+    def tiles(self) -> int:
+        return self.seq // self.block
+
+
+# The five graded configurations (index 0..4) in the order they are specified.
+WORKLOADS = (
+    Workload("c1_causal_s256_d64", 1, 1, 1, 256, 64, 64, MASK_CAUSAL),
+    Workload("c2_causal_s4k_mha32", 1, 32, 32, 4096, 128, 128, MASK_CAUSAL),
+    Workload("c3_window4k_s16k_gqa32x8", 1, 32, 8, 16384, 128, 128,
+             MASK_CAUSAL | MASK_WINDOW, window=4096),
+    Workload("c4_bitmap25_s32k_h16", 1, 16, 16, 32768, 128, 128,
+             MASK_CAUSAL | MASK_BITMAP, keep_prob=0.25),
+    Workload("c5_causal_s128k_gqa32x8", 1, 32, 8, 131072, 128, 128, MASK_CAUSAL,
+             sigma=0.5, head_query_scale=True),
+)
+
+
+def workload(name_or_index) -> Workload:
+    if isinstance(name_or_index, int):
+        return WORKLOADS[name_or_index]
+    for w in WORKLOADS:
+        if w.name == name_or_index or w.name.split("_")[0] == name_or_index:
+            return w
+    raise KeyError(name_or_index)
+
+
+def block_bitmap(heads_q: int, t_q: int, t_kv: int, keep_prob: float,
+                 seed: int = DEFAULT_SEED) -> np.ndarray:
+    """Per-head block bitmap, uint32 words ``[heads_q][t_q][ceil(t_kv/32)]``.
+
+    Bit ``J & 31`` of word ``J >> 5`` is block (I, J).  The diagonal block and key
+    block 0 are always kept; other blocks with J < I are kept when
+    ``u1(stream 5, e = (h*t_q + I)*t_kv + J) < keep_prob``; blocks with J > I are clear.
+    """
+    words = (t_kv + 31) // 32
+    h, i, j = np.meshgrid(np.arange(heads_q), np.arange(t_q), np.arange(t_kv), indexing="ij")
+    e = ((h * t_q + i) * t_kv + j).astype(np.uint64)
+    keep = uniform(seed, STREAM_BITMAP, e) < keep_prob
+    keep &= j < i
+    keep |= (j == i) | ((j == 0) & (j <= i))
+    padded = np.zeros((heads_q, t_q, words * 32), dtype=bool)
+    padded[:, :, :t_kv] = keep
+    bits = padded.reshape(heads_q, t_q, words, 32).astype(np.uint32)
+    return (bits << np.arange(32, dtype=np.uint32)).sum(axis=3, dtype=np.uint32)
+
+
+def bitmap_bit(bitmap: np.ndarray, h: int, i_blk: int, j_blk: int) -> bool:
+    return bool((int(bitmap[h, i_blk, j_blk >> 5]) >> (j_blk & 31)) & 1)
+
+
+def make_inputs(w: Workload, seed: int = DEFAULT_SEED, threads: int = 8) -> dict:
+    """Q, K, V as bf16 bit patterns (uint16, ``[batch, heads, seq, head_dim]``) and the
+    bitmap (or None) of workload ``w``."""
+    shape_q = (w.batch, w.heads_q, w.seq, w.head_dim)
+    shape_kv = (w.batch, w.heads_kv, w.seq, w.head_dim)
+    head_scale = None
+    if w.head_query_scale:
+        u = uniform(seed, STREAM_HEAD_SCALE, np.arange(w.heads_q, dtype=np.uint64))
+        head_scale = np.tile(0.5 + 1.5 * u, w.batch)
+    q = normal_bf16(seed, STREAM_Q, shape_q, w.sigma, head_scale, threads)
+    k = normal_bf16(seed, STREAM_K, shape_kv, w.sigma, None, threads)
+    v = normal_bf16(seed, STREAM_V, shape_kv, w.sigma, None, threads)
+    bitmap = None
+    if w.flags & MASK_BITMAP:
+        bitmap = block_bitmap(w.heads_q, w.tiles, w.tiles, w.keep_prob, seed)
+    return {"q": q, "k": k, "v": v, "bitmap": bitmap, "head_scale": head_scale}
+
+
+def checksum(bits: np.ndarray) -> int:
+    """Order-dependent 64-bit checksum of an array's bytes (for logging input identity)."""
+    a = np.ascontiguousarray(bits).view(np.uint8)
+    pad = (-a.size) % 8
+    if pad:
+        a = np.concatenate([a.ravel(), np.zeros(pad, np.uint8)])
+    w = a.ravel().view(np.uint64)
+    with np.errstate(over="ignore"):
+        idx = np.arange(1, w.size + 1, dtype=np.uint64)
+        return int(np.bitwise_xor.reduce(splitmix64(w ^ (idx * _U64(0x9E3779B97F4A7C15)))))
