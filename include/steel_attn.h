@@ -1,0 +1,151 @@
+/*
+ * steel_attn.h — C ABI of the block-sparse fused prefill attention library for NVIDIA B200.
+ *
+ * The operation (paper Eq. 1, generalised by `scale` and a mask): for every batch b, query
+ * head h and query row i,
+ *
+ *     O[b,h,i,:] = softmax_j( scale * Q[b,h,i,:] . K[b,g,j,:] + M[h,i,j] ) V[b,g,:,:]
+ *     LSE[b,h,i] = ln sum_j exp( scale * Q[b,h,i,:] . K[b,g,j,:] + M[h,i,j] )
+ *
+ * with g = h / (heads_q / heads_kv) (grouped-query attention, contiguous groups) and
+ * M = 0 where key j is visible to query i, -inf elsewhere.  It is computed as the paper's
+ * Algorithm 1: tiled Q K^T, online softmax (running row maximum m and row sum l), P V
+ * accumulation, final division by l — never materialising the score matrix, and following
+ * the paper's three mask cases (Sec. "The STEEL Pipeline"): a (query-tile, key-tile) pair
+ * whose elements are all masked is skipped (no memory traffic, no MMA), an unmasked pair is
+ * processed as is, a partially masked pair has the mask generated from coordinates on chip.
+ * The mask is never read from memory by the kernel; only a per-CTA work list derived from it.
+ *
+ * Visibility predicate (AND of the enabled terms; `off` = seq_kv - seq_q):
+ *     CAUSAL : j <= i + off
+ *     WINDOW : (i + off) - j < window          (with CAUSAL: exactly `window` keys incl. self)
+ *     BITMAP : bit (J & 31) of bitmap[(h * T_q + I) * ceil(T_kv / 32) + (J >> 5)] is set,
+ *              I = i / block_q, J = j / block_kv, T_q = ceil(seq_q / block_q), T_kv likewise.
+ * A query row with no visible key gets O = 0 and LSE = -inf.
+ *
+ * Memory layout: Q and O are [batch, heads_q, seq_q, head_dim], K and V are
+ * [batch, heads_kv, seq_kv, head_dim], all contiguous bfloat16; LSE is
+ * [batch, heads_q, seq_q] float32.  Arithmetic: bf16 operands, fp32 accumulation and
+ * softmax statistics; P is rounded to bf16 for the second product, l sums the unrounded P.
+ *
+ * Ownership and threading: every tensor pointer is a DEVICE pointer owned by the caller,
+ * 16-byte aligned, and must stay valid until the stream has executed the call.  The bitmap
+ * is a HOST pointer read only during steel_attn_create.  A handle owns its device work lists
+ * and scheduler counter; it is bound to the device that was current at create time and must
+ * not be used by two streams at once.  All functions return a status code; nothing throws,
+ * aborts or traps.  There is no CPU fallback: without a usable CUDA device the run fails.
+ */
+#ifndef STEEL_ATTN_H_
+#define STEEL_ATTN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct steel_attn steel_attn_t; /* opaque, owned by the library */
+
+typedef enum {
+  STEEL_OK = 0,
+  STEEL_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer, bad flags */
+  STEEL_ERR_UNSUPPORTED = 2, /* valid problem outside this build's limits (see create)         */
+  STEEL_ERR_ALLOC = 3,       /* host or device allocation failed                               */
+  STEEL_ERR_CUDA = 4,        /* a CUDA call failed (no device, wrong architecture, launch)     */
+  STEEL_ERR_TIMEOUT = 5      /* a bounded device-side wait expired; outputs are undefined      */
+} steel_status_t;
+
+enum { STEEL_MASK_CAUSAL = 1u, STEEL_MASK_WINDOW = 2u, STEEL_MASK_BITMAP = 4u };
+
+typedef struct {
+  uint32_t flags;           /* OR of STEEL_MASK_*; 0 = dense attention                         */
+  int32_t block_q;          /* mask block sizes in tokens, 64 or 128 (0 = 128); they define the */
+  int32_t block_kv;         /* BITMAP grid and the granularity at which tiles are counted       */
+  int64_t window;           /* W > 0 tokens, used iff WINDOW                                    */
+  const uint32_t *bitmap;   /* HOST pointer, used iff BITMAP, copied by create;                 */
+                            /* [heads_q][T_q][ceil(T_kv/32)] words, shared across the batch     */
+} steel_mask_desc_t;
+
+typedef struct {
+  int32_t batch, heads_q, heads_kv; /* heads_q % heads_kv == 0                                  */
+  int32_t seq_q, seq_kv;            /* any positive lengths (ragged last tiles are masked)       */
+  int32_t head_dim;                 /* 64 or 128                                                 */
+  float scale;                      /* finite, > 0; multiplies q.k before softmax                */
+  steel_mask_desc_t mask;
+} steel_attn_params_t;
+
+/* Work-list statistics of a plan (the skip set of the three mask cases, at the kernel's
+ * 128 x 128 tile granularity). */
+typedef struct {
+  int64_t kept_tiles;     /* (query-block, key-block) pairs that are not fully masked, counted  */
+                          /* at the descriptor's block_q x block_kv granularity                 */
+  int64_t partial_tiles;  /* of those, pairs with some masked element                           */
+  int64_t total_tiles;    /* all block pairs of the problem, skipped ones included              */
+  int64_t exec_tiles;     /* 128 x 128 kernel tiles executed (equals kept_tiles for 128 blocks)  */
+  int64_t exec_partial;   /* of those, tiles on which the element-wise mask is applied          */
+  int64_t work_items;     /* scheduler items (one or two query tiles that share key loads)      */
+  int64_t steps;          /* key-tile steps summed over items                                   */
+  int64_t kv_tile_loads;  /* K (equally V) tile loads issued; exec_tiles minus shared loads     */
+  int64_t list_entries;   /* explicit step-list entries held in device memory (bitmap masks)    */
+  int64_t max_cta_steps;  /* steps of the most loaded persistent CTA                            */
+  int64_t grid;           /* persistent CTAs launched                                           */
+  double effective_flop;  /* 4 * block_q * block_kv * head_dim * kept_tiles                     */
+  double useful_flop;     /* 4 * head_dim * (number of visible (i, j) pairs)                     */
+} steel_attn_stats_t;
+
+/*
+ * Validate `params`, classify every tile (mask cases i-iii), build the work items and their
+ * key-tile lists, order them for the persistent scheduler and upload them to the current
+ * CUDA device.  On success *out receives the handle; on failure *out is NULL.
+ * STEEL_ERR_UNSUPPORTED: head_dim not in {64, 128}; block sizes other than 64 or 128 or
+ * block_q != block_kv; more than 2^24 key tiles; batch * heads * seq beyond 2^31 rows.  Allocates device memory;
+ * synchronises the device once.
+ */
+steel_status_t steel_attn_create(const steel_attn_params_t *params, steel_attn_t **out);
+
+/*
+ * Enqueue one attention call on `cuda_stream` (a cudaStream_t cast to void*; NULL = default
+ * stream).  q, k, v, o: device bf16 tensors in the layouts above; lse: device float32 or
+ * NULL.  Asynchronous: no allocation, no host synchronisation.  One persistent kernel is
+ * launched; device-side waits are bounded and, if one expires, the kernel stops and the
+ * error is reported by steel_attn_last_status.
+ */
+steel_status_t steel_attn_run(steel_attn_t *handle, const void *q, const void *k, const void *v,
+                              void *o, float *lse, void *cuda_stream);
+
+/*
+ * Synchronise `cuda_stream` and report the device-side status word of the handle's last
+ * runs (STEEL_OK or STEEL_ERR_TIMEOUT), then clear it.
+ */
+steel_status_t steel_attn_last_status(steel_attn_t *handle, void *cuda_stream);
+
+/* Release the handle and its device memory.  destroy(NULL) is STEEL_OK. */
+steel_status_t steel_attn_destroy(steel_attn_t *handle);
+
+/* Statistics of the handle's plan. */
+steel_status_t steel_attn_get_stats(const steel_attn_t *handle, steel_attn_stats_t *stats);
+
+/*
+ * Host-only planning: the same validation, tile classification and work-list construction as
+ * steel_attn_create, without touching CUDA.  `stats` receives the statistics.  If `tiles` is
+ * not NULL it receives, for every executed pair in the order the kernel's roles walk them,
+ * six int32 values {item, batch, head, query_tile, key_tile, flags} (tiles are 128 x 128;
+ * flags bit 0: partial, bit 1: the K/V load is shared with the item's other query tile,
+ * bits 4..7: enabled 64x64 sub-blocks TL, TR, BL, BR), up to `capacity` records; *n_tiles receives the number written.
+ */
+steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_attn_stats_t *stats,
+                                    int32_t *tiles, int64_t capacity, int64_t *n_tiles);
+
+/* Number of scheduler policies and selection of one for subsequently created handles
+ * (process-wide; default 0).  0: query tiles paired for shared K/V loads, items ordered
+ * KV-head-major then longest first (the sparsity-aware placement idea of the paper's Sec.
+ * "Sparsity-Aware Pipeline Placement" recast for persistent CTAs); 1: same items in natural
+ * (uniform, contiguous) order. */
+steel_status_t steel_attn_set_policy(int32_t policy);
+
+const char *steel_status_string(steel_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STEEL_ATTN_H_ */
