@@ -16,7 +16,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -50,29 +49,36 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the clock-event (throttle) reasons through NVML (read-only queries)
+    every few milliseconds while the timed region runs."""
 
-    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
 
-    def __init__(self, index: int):
-        self.index = index
-        self.samples = []
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.sm, self.mask, self.max_mhz, self.error = [], 0, None, None
         self._stop = threading.Event()
         self._thread = threading.Thread(target=self._run, daemon=True)
 
     def _run(self):
-        while not self._stop.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True,
-                                     timeout=5).stdout.strip()
-                if out:
-                    self.samples.append([x.strip() for x in out.split(",")])
-            except Exception:
-                pass
-            self._stop.wait(0.1)
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if visible:
+                ids = [x for x in visible.split(",") if x]
+                if idx < len(ids) and ids[idx].isdigit():
+                    idx = int(ids[idx])
+            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                self.mask |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                self._stop.wait(self.period)
+        except Exception as exc:  # report, never fail the benchmark on a monitoring problem
+            self.error = repr(exc)
 
     def __enter__(self):
         self._thread.start()
@@ -83,13 +89,12 @@ class ClockSampler:
         self._thread.join(timeout=10)
 
     def summary(self) -> dict:
-        sm = [float(s[0]) for s in self.samples if s and s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if len(s) > 1 and s[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names)
-                   if any(len(s) > 2 + i and s[2 + i].lower().startswith("active") for s in self.samples)]
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.samples)}
+        out = {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+               "sm_min_mhz": min(self.sm) if self.sm else None,
+               "reasons": [n for bit, n in self.REASONS.items() if self.mask & bit], "samples": len(self.sm)}
+        if self.error:
+            out["error"] = self.error
+        return out
 
 
 def oracle_sample_rows(w, n_rows: int, seed: int = 7) -> np.ndarray:
@@ -162,6 +167,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--policy", type=int, default=0)
+    ap.add_argument("--profile-heads", type=int, default=0,
+                    help="shrink the workload to this many query heads (same KV grouping) for ncu captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "steel" else args.warmup
 
@@ -169,6 +176,11 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     w = inputs.workload(int(args.workload) if args.workload.isdigit() else args.workload)
+    if args.profile_heads:
+        import dataclasses
+        group = w.heads_q // w.heads_kv
+        w = dataclasses.replace(w, name=f"{w.name}_h{args.profile_heads}", heads_q=args.profile_heads,
+                                heads_kv=max(1, args.profile_heads // group))
 
     if args.impl == "reference":
         run_reference(args, w, rank, world)

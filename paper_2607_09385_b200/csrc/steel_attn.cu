@@ -22,6 +22,7 @@ struct steel_attn {
   int32_t *d_cta_begin = nullptr;
   StepPair *d_steps = nullptr;
   int32_t *d_status = nullptr;
+  long long *d_trace = nullptr;  // debug builds only
 };
 
 namespace {
@@ -158,6 +159,7 @@ steel_status_t steel_attn_run(steel_attn_t *h, const void *q, const void *k, con
   kp.window = int32_t(p.mask.window > std::numeric_limits<int32_t>::max() ? std::numeric_limits<int32_t>::max()
                                                                           : p.mask.window);
   kp.scale_log2 = p.scale * 1.4426950408889634f;
+  kp.trace = h->d_trace;
   if (launch_attention(p.head_dim, map_q, map_k, map_v, kp, h->grid, static_cast<cudaStream_t>(cuda_stream)) !=
       cudaSuccess)
     return STEEL_ERR_CUDA;
@@ -219,6 +221,15 @@ steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_att
   if (n_tiles) *n_tiles = n;
   return STEEL_OK;
 }
+
+#ifdef STEEL_TRACE
+// Debug builds: device buffer of gridDim.x * 32 counters filled by the kernel's roles.
+steel_status_t steel_attn_set_trace(steel_attn_t *h, long long *device_buffer) {
+  if (!h) return STEEL_ERR_INVALID_ARG;
+  h->d_trace = device_buffer;
+  return STEEL_OK;
+}
+#endif
 
 steel_status_t steel_attn_set_policy(int32_t policy) {
   if (policy < 0 || policy > 1) return STEEL_ERR_INVALID_ARG;

@@ -1,23 +1,24 @@
 // Fused block-sparse attention kernel for sm_100a (paper Algorithm 1 on one persistent CTA per SM).
 //
 // A CTA processes work items; an item is one or two query tiles (128 rows each, "slots") that walk
-// the same sequence of key-tile steps.  Roles:
+// the same sequence of key-tile steps.  Roles (three warpgroups, register file re-split between them):
 //   warps 0-3 / 4-7 : softmax warpgroup of slot 0 / 1.  Thread r owns query row r: it reads the
 //                     score row S (fp32) from TMEM, applies scale and (partial tiles only) the mask
 //                     computed from coordinates, keeps the running maximum m and sum l, writes
-//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S, rescales O when the
-//                     maximum has grown, and at the end writes O / l and LSE.  (Algorithm 1, First
-//                     Stage's scale_and_mask and rowmax, Second Stage, and the rescale of the Third.)
+//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S (in two halves, so the
+//                     second product can start on the first), rescales O when the maximum has grown,
+//                     and at the end writes O / l and LSE.  (Algorithm 1: scale_and_mask and rowmax of
+//                     the First Stage, the Second Stage, and the rescale of the Third.)
 //   warp 8          : TMA producer.  Loads Q once per item and K_j / V_j for executed tiles only into
 //                     a shared-memory ring; a tile wanted by both slots in the same step is loaded once.
 //   warp 9          : MMA issuer.  S = Q K^T (both operands in shared memory) and O += P V (P from
 //                     TMEM, V from shared memory) on tcgen05 with fp32 accumulators in TMEM.
-// All three walk an item's steps with the same generator (walk_item), so ring positions agree
-// without communication.  Every mbarrier wait is bounded; on expiry the CTA sets the status word
-// and all roles leave.
+// Producer and MMA issuer enumerate an item's operations with the same generator (Walker), so ring
+// positions agree without communication.  Every mbarrier wait is bounded; on expiry the CTA sets
+// the status word and all roles leave.
 #include <cuda.h>
-#include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_runtime.h>
 #include <math_constants.h>
 
 #include "sm100_ptx.cuh"
@@ -26,12 +27,15 @@
 
 namespace steel {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;        // softmax slot 0, softmax slot 1, {producer, MMA, 2 idle warps}
+constexpr int kRegsSoftmax = 216;    // registers per thread after the warpgroups re-split the file
+constexpr int kRegsOther = 72;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr long long kTimeoutCycles = 4000000000ll;  // about two seconds
 constexpr float kRescaleThreshold = 8.0f;           // lazy rescale: P stays below 2^8
 constexpr int kMaxStages = 10;
+constexpr int kFifoDepth = 32;
 constexpr uint32_t kMaskCausal = 1u, kMaskWindow = 2u;
 
 template <int D>
@@ -47,10 +51,32 @@ struct Cfg {
 
 struct Ctrl {
   uint64_t ring_full[kMaxStages], ring_empty[kMaxStages];
-  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2], o_empty[2];
+  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2][2], o_full[2], o_empty[2];
+  uint32_t fifo[kFifoDepth];  // command words from the producer to the MMA issuer (0 = empty)
   uint32_t tmem_base;
   int abort;
 };
+
+// Command word layout (producer -> MMA issuer).
+constexpr uint32_t kCmdValid = 1u << 0, kCmdIsS = 1u << 1, kCmdSlot1 = 1u << 2, kCmdRingShift = 3,  // 4 bits
+                   kCmdRingPhase = 1u << 7, kCmdWaitFirst = 1u << 8, kCmdFirstPhase = 1u << 9,
+                   kCmdFinalUse = 1u << 10, kCmdEnd = 1u << 11, kCmdAcc = 1u << 12, kCmdPPhase = 1u << 13,
+                   kCmdExit = 1u << 14;
+
+// Optional per-role wait accounting (compiled in with -DSTEEL_TRACE only): cycles per CTA, 32 slots.
+#ifdef STEEL_TRACE
+#define TRACE_T0() const long long trace_t0_ = clock64()
+#define TRACE_ADD(idx) trace_acc[idx] += clock64() - trace_t0_
+#define TRACE_DECL(n) long long trace_acc[n] = {}
+#define TRACE_FLUSH(base, n)                                                               \
+  if (p.trace)                                                                             \
+    for (int i_ = 0; i_ < (n); ++i_) p.trace[size_t(blockIdx.x) * 32 + (base) + i_] = trace_acc[i_]
+#else
+#define TRACE_T0()
+#define TRACE_ADD(idx)
+#define TRACE_DECL(n)
+#define TRACE_FLUSH(base, n)
+#endif
 
 __device__ __forceinline__ bool bounded_wait(uint64_t *bar, uint32_t parity, Ctrl &ctrl, int32_t *status) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -69,133 +95,224 @@ __device__ __forceinline__ bool bounded_wait(uint64_t *bar, uint32_t parity, Ctr
   }
 }
 
-__device__ __forceinline__ WorkItem load_item(const WorkItem *items, int k) {
-  WorkItem w;
+// A work item unpacked into scalars (no indexable arrays, so everything stays in registers).
+struct Item {
+  int batch, kv_head, head0, head1, qtile0, qtile1, lo0, lo1, hi0, hi1, n_steps, kind, j0, list_off;
+  __device__ __forceinline__ int lo(int s) const { return s ? lo1 : lo0; }
+  __device__ __forceinline__ int hi(int s) const { return s ? hi1 : hi0; }
+  __device__ __forceinline__ int head(int s) const { return s ? head1 : head0; }
+  __device__ __forceinline__ int qtile(int s) const { return s ? qtile1 : qtile0; }
+  __device__ __forceinline__ bool active(int s) const { return head(s) >= 0 && hi(s) >= lo(s); }
+};
+
+__device__ __forceinline__ Item load_item(const WorkItem *items, int k) {
   const int4 *src = reinterpret_cast<const int4 *>(items + k);
-  int4 *dst = reinterpret_cast<int4 *>(&w);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) dst[i] = __ldg(src + i);
+  const int4 a = __ldg(src), b = __ldg(src + 1), c = __ldg(src + 2), d = __ldg(src + 3);
+  Item w;
+  w.batch = a.x;  w.kv_head = a.y;  w.head0 = a.z;  w.head1 = a.w;
+  w.qtile0 = b.x; w.qtile1 = b.y;   w.lo0 = b.z;    w.lo1 = b.w;
+  w.hi0 = c.x;    w.hi1 = c.y;      w.n_steps = c.z; w.kind = c.w;
+  w.j0 = d.x;     w.list_off = d.y;
   return w;
 }
 
-__device__ __forceinline__ bool slot_active(const WorkItem &w, int s) { return w.head[s] >= 0 && w.hi[s] >= w.lo[s]; }
-
 // Entries {slot 0, slot 1} of step t: key-tile index plus the present bit (0 when the slot is absent).
-__device__ __forceinline__ uint2 load_step(const WorkItem &w, const StepPair *steps, int t) {
+__device__ __forceinline__ uint2 load_step(const Item &w, const StepPair *steps, int t) {
   uint2 e = make_uint2(0u, 0u);
   if (t >= w.n_steps) return e;
   if (w.kind == 0) {
-    uint32_t v = uint32_t(w.j0 + t) | kEntryPresent;
-    if (slot_active(w, 0) && t >= w.lo[0] && t <= w.hi[0]) e.x = v;
-    if (slot_active(w, 1) && t >= w.lo[1] && t <= w.hi[1]) e.y = v;
+    const uint32_t v = uint32_t(w.j0 + t) | kEntryPresent;
+    if (w.active(0) && t >= w.lo0 && t <= w.hi0) e.x = v;
+    if (w.active(1) && t >= w.lo1 && t <= w.hi1) e.y = v;
   } else {
     e = __ldg(reinterpret_cast<const uint2 *>(steps + w.list_off + t));
   }
   return e;
 }
 
-// The canonical order of an item's tensor-core operations, shared by the producer (which loads a
-// tile at its first use) and the MMA issuer.  For each step t: first S(s, t) of slots that start
-// at t, then for each present slot PV(s, t) followed by S(s, t + 1).  `entry` numbers ring fills;
-// a tile wanted by both slots in one step is filled once (slot 0 first, slot 1 last).
-template <class OpS, class OpPV>
-__device__ __forceinline__ void walk_item(const WorkItem &w, const StepPair *steps, uint32_t &ring_pos, OpS &&op_s,
-                                          OpPV &&op_pv, bool &ok) {
-  uint32_t last_k = 0, last_v = 0;
-  uint2 cur = load_step(w, steps, 0), nxt;
-  auto ent = [](const uint2 &e, int s) { return s == 0 ? e.x : e.y; };
-  auto visit = [&](const uint2 &e, int s, int t, bool is_s) {
-    const uint32_t mine = ent(e, s), other = ent(e, 1 - s);
-    const bool shared = other != 0 && ((mine ^ other) & kEntryTileMask) == 0;
-    uint32_t &last = is_s ? last_k : last_v;
-    uint32_t entry;
-    bool first, final_use;
-    if (s == 0) {
-      entry = ring_pos++;
-      last = entry;
-      first = true;
-      final_use = !shared;
-    } else if (shared) {
-      entry = last;
-      first = false;
-      final_use = true;
-    } else {
-      entry = ring_pos++;
-      first = true;
-      final_use = true;
+// The canonical order of an item's tensor-core operations S(s, t) = Q_s K_j^T and PV(s, t):
+// O_s += P_s V_j, shared by the producer (which loads a tile at its first use) and the MMA issuer.
+// For each step t: first S(s, t) of slots that start at t, then for each present slot PV(s, t)
+// followed by S(s, t + 1).  A tile wanted by both slots in one step is one ring fill: slot 0 uses
+// it first, slot 1 last (the planner guarantees lo0 <= lo1).  `ring` counts fills.
+// op(s, t, j, is_s, fill, first, last) returns false to stop.
+struct RingPos {
+  uint32_t slot, phase;  // next fill goes to `slot`; `phase` flips each time the ring wraps
+};
+struct Fill {
+  uint32_t slot, phase;
+};
+
+template <int kStages, class Op>
+__device__ __forceinline__ bool walk_item(const Item &w, const StepPair *steps, RingPos &ring, Op &&op) {
+  Fill last_k{0, 0}, last_v{0, 0};
+  auto take = [&]() {
+    Fill f{ring.slot, ring.phase};
+    if (++ring.slot == uint32_t(kStages)) {
+      ring.slot = 0;
+      ring.phase ^= 1u;
     }
-    const int j = int(mine & kEntryTileMask);
-    if (is_s) ok = op_s(s, t, j, entry, first, final_use);
-    else ok = op_pv(s, t, j, entry, first, final_use);
+    return f;
   };
-  for (int t = 0; t < w.n_steps && ok; ++t) {
-    nxt = load_step(w, steps, t + 1);
-#pragma unroll
-    for (int s = 0; s < 2; ++s)
-      if (ok && ent(cur, s) != 0 && t == w.lo[s]) visit(cur, s, t, true);
-#pragma unroll
-    for (int s = 0; s < 2; ++s)
-      if (ok && ent(cur, s) != 0) {
-        visit(cur, s, t, false);
-        if (ok && t < w.hi[s]) visit(nxt, s, t + 1, true);
+  auto visit = [&](const uint2 &e, int s, int t, bool is_s) -> bool {
+    const uint32_t mine = s ? e.y : e.x, other = s ? e.x : e.y;
+    const bool shared = other != 0 && ((mine ^ other) & kEntryTileMask) == 0;
+    Fill &last = is_s ? last_k : last_v;
+    Fill f;
+    bool first = true, final_use = true;
+    if (s == 1 && shared) {
+      f = last;
+      first = false;
+    } else {
+      f = take();
+      if (s == 0) {
+        last = f;
+        final_use = !shared;
       }
+    }
+    return op(s, t, int(mine & kEntryTileMask), is_s, f, first, final_use);
+  };
+  uint2 cur = load_step(w, steps, 0);
+  for (int t = 0; t < w.n_steps; ++t) {
+    const uint2 nxt = load_step(w, steps, t + 1);
+    if (cur.x != 0 && t == w.lo0 && !visit(cur, 0, t, true)) return false;
+    if (cur.y != 0 && t == w.lo1 && !visit(cur, 1, t, true)) return false;
+    if (cur.x != 0) {
+      if (!visit(cur, 0, t, false)) return false;
+      if (t < w.hi0 && !visit(nxt, 0, t + 1, true)) return false;
+    }
+    if (cur.y != 0) {
+      if (!visit(cur, 1, t, false)) return false;
+      if (t < w.hi1 && !visit(nxt, 1, t + 1, true)) return false;
+    }
     cur = nxt;
   }
+  return true;
 }
 
 // ------------------------------------------------------------------------------------------------
+// Bounded push / pop of the single-producer single-consumer command queue in shared memory.
+__device__ __forceinline__ bool fifo_push(Ctrl &ctrl, uint32_t &tail, uint32_t word, int32_t *status) {
+  volatile uint32_t *cell = &ctrl.fifo[tail];
+  if (*cell != 0) {
+    const long long start = clock64();
+    uint32_t n = 0;
+    while (*cell != 0) {
+      if ((++n & 63u) == 0) {
+        if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return false;
+        if (clock64() - start > kTimeoutCycles) {
+          *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
+          atomicExch(status, 5);
+          return false;
+        }
+      }
+    }
+  }
+  *cell = word;
+  tail = (tail + 1) & (kFifoDepth - 1);
+  return true;
+}
+__device__ __forceinline__ uint32_t fifo_pop(Ctrl &ctrl, uint32_t &head, int32_t *status) {
+  volatile uint32_t *cell = &ctrl.fifo[head];
+  uint32_t word = *cell;
+  if (word == 0) {
+    const long long start = clock64();
+    uint32_t n = 0;
+    while ((word = *cell) == 0) {
+      if ((++n & 63u) == 0) {
+        if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return kCmdExit;
+        if (clock64() - start > kTimeoutCycles) {
+          *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
+          atomicExch(status, 5);
+          return kCmdExit;
+        }
+      }
+    }
+  }
+  *cell = 0;
+  head = (head + 1) & (kFifoDepth - 1);
+  return word;
+}
+
+// The producer is also the scheduler: it walks the items, issues the TMA loads and publishes one
+// command word per tensor-core operation, so the MMA issuer's own loop stays a few instructions long.
 template <int D>
 __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, const CUtensorMap *map_k,
                               const CUtensorMap *map_v, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring) {
   using C = Cfg<D>;
-  uint32_t ring_pos = 0, n_use[2] = {0, 0}, q_issued[2] = {0, 0};
+  RingPos ring{0, 0};
+  uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, fills = 0, tail = 0;
   bool ok = true;
-  auto load_tile = [&](const CUtensorMap *map, int j, int z, uint32_t entry) -> bool {
-    const uint32_t slot = entry % C::kStages, fill = entry / C::kStages;
-    if (!bounded_wait(&ctrl.ring_empty[slot], (fill & 1u) ^ 1u, ctrl, p.status)) return false;
-    mbar_arrive_expect_tx(&ctrl.ring_full[slot], C::kTileBytes);
-#pragma unroll
-    for (int b = 0; b < C::kBoxes; ++b)
-      tma_load_3d(smem_ring + slot * C::kTileBytes + b * C::kBoxBytes, map, &ctrl.ring_full[slot], b * 64, j * kTile, z);
-    return true;
-  };
   const int k_end = p.cta_begin[blockIdx.x + 1];
   for (int k = p.cta_begin[blockIdx.x]; k < k_end && ok; ++k) {
-    const WorkItem w = load_item(p.items, k);
-    for (int s = 0; s < 2 && ok; ++s) {
-      if (!slot_active(w, s)) continue;
-      ok = bounded_wait(&ctrl.q_empty[s], (n_use[s] & 1u) ^ 1u, ctrl, p.status);
+    const Item w = load_item(p.items, k);
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      if (!ok || !w.active(s)) continue;
+      uint32_t &n_use = s ? n_use1 : n_use0;
+      ok = bounded_wait(&ctrl.q_empty[s], (n_use & 1u) ^ 1u, ctrl, p.status);
       if (!ok) break;
       mbar_arrive_expect_tx(&ctrl.q_full[s], C::kTileBytes);
 #pragma unroll
       for (int b = 0; b < C::kBoxes; ++b)
         tma_load_3d(smem_q + s * C::kTileBytes + b * C::kBoxBytes, map_q, &ctrl.q_full[s], b * 64,
-                    w.qtile[s] * kTile, w.batch * p.heads_q + w.head[s]);
-      ++n_use[s];
-      q_issued[s] = n_use[s];
+                    w.qtile(s) * kTile, w.batch * p.heads_q + w.head(s));
+      ++n_use;
     }
+    if (!ok) break;
     const int z = w.batch * p.heads_kv + w.kv_head;
-    walk_item(
-        w, p.steps, ring_pos,
-        [&](int, int, int j, uint32_t entry, bool first, bool) { return first ? load_tile(map_k, j, z, entry) : true; },
-        [&](int, int, int j, uint32_t entry, bool first, bool) { return first ? load_tile(map_v, j, z, entry) : true; },
-        ok);
+    ok = walk_item<C::kStages>(w, p.steps, ring, [&](int s, int t, int j, bool is_s, Fill f, bool first, bool final_use) -> bool {
+      if (first) {
+        if (!bounded_wait(&ctrl.ring_empty[f.slot], f.phase ^ 1u, ctrl, p.status)) return false;
+        mbar_arrive_expect_tx(&ctrl.ring_full[f.slot], C::kTileBytes);
+        const CUtensorMap *map = is_s ? map_k : map_v;
+#pragma unroll
+        for (int b = 0; b < C::kBoxes; ++b)
+          tma_load_3d(smem_ring + f.slot * C::kTileBytes + b * C::kBoxBytes, map, &ctrl.ring_full[f.slot], b * 64,
+                      j * kTile, z);
+        ++fills;
+      }
+      // phase of this item's use of the slot: Q-full for S, O-empty (inverted) for PV
+      const uint32_t use_phase = ((s ? n_use1 : n_use0) - 1u) & 1u;
+      uint32_t cmd = kCmdValid | (f.slot << kCmdRingShift) | (f.phase ? kCmdRingPhase : 0u) |
+                     (s ? kCmdSlot1 : 0u) | (final_use ? kCmdFinalUse : 0u);
+      if (t == w.lo(s)) cmd |= kCmdWaitFirst;
+      if (t == w.hi(s)) cmd |= kCmdEnd;
+      if (is_s) {
+        cmd |= kCmdIsS | (use_phase ? kCmdFirstPhase : 0u);
+      } else {
+        uint32_t &n_sp = s ? n_sp1 : n_sp0;
+        cmd |= ((use_phase ^ 1u) ? kCmdFirstPhase : 0u) | (t > w.lo(s) ? kCmdAcc : 0u) | ((n_sp & 1u) ? kCmdPPhase : 0u);
+        ++n_sp;
+      }
+      return fifo_push(ctrl, tail, cmd, p.status);
+    });
   }
+  if (ok) ok = fifo_push(ctrl, tail, kCmdValid | kCmdExit, p.status);
   if (!ok) {
     // leave only after the copies already issued have landed (bounded), so none writes into
-    // shared memory of a later CTA
-    const uint32_t first = ring_pos > uint32_t(C::kStages) ? ring_pos - C::kStages : 0;
-    for (uint32_t e = first; e < ring_pos; ++e) {
+    // shared memory of a later CTA: the last min(fills, stages) fills end at ring.slot - 1
+    const uint32_t pending = fills < uint32_t(C::kStages) ? fills : uint32_t(C::kStages);
+    uint32_t slot = ring.slot, phase = ring.phase;
+    for (uint32_t e = 0; e < pending; ++e) {
+      if (slot == 0) {
+        slot = C::kStages;
+        phase ^= 1u;
+      }
+      --slot;
       const long long start = clock64();
-      while (!mbar_try_wait(&ctrl.ring_full[e % C::kStages], (e / C::kStages) & 1u) && clock64() - start < kTimeoutCycles / 8) {
+      while (!mbar_try_wait(&ctrl.ring_full[slot], phase) && clock64() - start < kTimeoutCycles / 8) {
       }
     }
-    for (int s = 0; s < 2; ++s)
-      if (q_issued[s]) {
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const uint32_t n_use = s ? n_use1 : n_use0;
+      if (n_use) {
         const long long start = clock64();
-        while (!mbar_try_wait(&ctrl.q_full[s], (q_issued[s] - 1) & 1u) && clock64() - start < kTimeoutCycles / 8) {
+        while (!mbar_try_wait(&ctrl.q_full[s], (n_use - 1) & 1u) && clock64() - start < kTimeoutCycles / 8) {
         }
       }
+    }
   }
 }
 
@@ -211,100 +328,129 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
   const uint64_t desc_q0 = make_smem_desc(smem_u32(smem_q), 16, 1024);
   const uint64_t desc_k0 = make_smem_desc(smem_u32(smem_ring), 16, 1024);
   const uint64_t desc_v0 = make_smem_desc(smem_u32(smem_ring), C::kBoxBytes, 1024);
-  uint32_t ring_pos = 0, n_sp[2] = {0, 0}, n_use[2] = {0, 0};
-  bool ok = true;
-  const int k_end = p.cta_begin[blockIdx.x + 1];
-  for (int k = p.cta_begin[blockIdx.x]; k < k_end && ok; ++k) {
-    const WorkItem w = load_item(p.items, k);
-    walk_item(
-        w, p.steps, ring_pos,
-        [&](int s, int t, int, uint32_t entry, bool, bool final_use) -> bool {
-          const uint32_t slot = entry % C::kStages, fill = entry / C::kStages;
-          if (t == w.lo[s] && !bounded_wait(&ctrl.q_full[s], n_use[s] & 1u, ctrl, p.status)) return false;
-          if (!bounded_wait(&ctrl.ring_full[slot], fill & 1u, ctrl, p.status)) return false;
-          tc_fence_after();
-          const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
-          const uint64_t dk = desc_k0 + uint64_t((slot * C::kTileBytes) >> 4);
+  uint32_t head = 0;
+  while (true) {
+    const uint32_t cmd = fifo_pop(ctrl, head, p.status);
+    if (cmd & kCmdExit) break;
+    const uint32_t s = (cmd & kCmdSlot1) ? 1u : 0u;
+    const uint32_t slot = (cmd >> kCmdRingShift) & 0xFu, ring_phase = (cmd & kCmdRingPhase) ? 1u : 0u;
+    const uint32_t first_phase = (cmd & kCmdFirstPhase) ? 1u : 0u;
+    if (cmd & kCmdIsS) {
+      if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.q_full[s], first_phase, ctrl, p.status)) break;
+      if (!bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
+      tc_fence_after();
+      const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
+      const uint64_t dk = desc_k0 + uint64_t((slot * C::kTileBytes) >> 4);
+      const uint32_t t_s = tmem + C::kColS + s * kTile;
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
-            mma_ss(tmem + C::kColS + s * kTile, dq + off, dk + off, idesc_s, kk > 0);
-          }
-          tc_commit(&ctrl.s_full[s]);
-          if (final_use) tc_commit(&ctrl.ring_empty[slot]);
-          if (t == w.hi[s]) tc_commit(&ctrl.q_empty[s]);
-          return true;
-        },
-        [&](int s, int t, int, uint32_t entry, bool, bool final_use) -> bool {
-          const uint32_t slot = entry % C::kStages, fill = entry / C::kStages;
-          if (!bounded_wait(&ctrl.p_full[s], n_sp[s] & 1u, ctrl, p.status)) return false;
-          ++n_sp[s];
-          if (t == w.lo[s] && !bounded_wait(&ctrl.o_empty[s], (n_use[s] & 1u) ^ 1u, ctrl, p.status)) return false;
-          if (!bounded_wait(&ctrl.ring_full[slot], fill & 1u, ctrl, p.status)) return false;
-          tc_fence_after();
-          const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
+        mma_ss(t_s, dq + off, dk + off, idesc_s, kk > 0);
+      }
+      tc_commit(&ctrl.s_full[s]);
+      if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdEnd) tc_commit(&ctrl.q_empty[s]);
+    } else {
+      if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.o_empty[s], first_phase, ctrl, p.status)) break;
+      if (!bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
+      const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
+      const uint32_t t_o = tmem + C::kColO + s * D, t_p = tmem + C::kColS + s * kTile;
+      const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u, p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
+      bool ok = true;
 #pragma unroll
-          for (int kk = 0; kk < kTile / 16; ++kk)
-            mma_ts(tmem + C::kColO + s * D, tmem + C::kColS + s * kTile + kk * 8, dv + uint64_t((kk * 2048) >> 4),
-                   idesc_pv, (t > w.lo[s] || kk > 0) ? 1u : 0u);
-          if (final_use) tc_commit(&ctrl.ring_empty[slot]);
-          if (t == w.hi[s]) {
-            tc_commit(&ctrl.o_full[s]);
-            ++n_use[s];
-          }
-          return true;
-        },
-        ok);
+      for (int half = 0; half < 2; ++half) {
+        ok = bounded_wait(&ctrl.p_full[s][half], p_phase, ctrl, p.status);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
+          mma_ts(t_o, t_p + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+      }
+      if (!ok) break;
+      if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdEnd) tc_commit(&ctrl.o_full[s]);
+    }
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int D>
-__device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, const int r) {
+// exp2 of 64 scaled scores -> 32 packed bf16x2 registers; accumulates the row sum in two lanes pairs.
+__device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, float2 scale2, float2 neg_m2,
+                                         float2 &acc_a, float2 &acc_b, uint32_t (&packed)[32]) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    const int e = base + 2 * i;
+    float2 y0 = ffma2(make_float2(x[e], x[e + 1]), scale2, neg_m2);
+    float2 y1 = ffma2(make_float2(x[e + 2], x[e + 3]), scale2, neg_m2);
+    y0.x = ex2_approx(y0.x);
+    y0.y = ex2_approx(y0.y);
+    y1.x = ex2_approx(y1.x);
+    y1.y = ex2_approx(y1.y);
+    acc_a = fadd2(acc_a, y0);
+    acc_b = fadd2(acc_b, y1);
+    packed[i] = pack_bf16x2(y0.x, y0.y);
+    packed[i + 1] = pack_bf16x2(y1.x, y1.y);
+  }
+}
+
+template <int D, int s>
+__device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int r) {
   using C = Cfg<D>;
+  const int lane = r % 32;
   const uint32_t lane_base = uint32_t((r / 32) * 32) << 16;
   const uint32_t t_s = ctrl.tmem_base + lane_base + C::kColS + s * kTile;
   const uint32_t t_o = ctrl.tmem_base + lane_base + C::kColO + s * D;
   const bool causal = (p.mask_flags & kMaskCausal) != 0, windowed = (p.mask_flags & kMaskWindow) != 0;
   const int off = p.seq_kv - p.seq_q;
   const float scale_log2 = p.scale_log2;
+  const float2 scale2 = make_float2(scale_log2, scale_log2);
   __nv_bfloat16 *o_base = static_cast<__nv_bfloat16 *>(p.o);
   uint32_t n_sp = 0, n_use = 0;
+  TRACE_DECL(7);
+#ifdef STEEL_TRACE
+  const long long role_t0 = clock64();
+#endif
 
   const int k_end = p.cta_begin[blockIdx.x + 1];
   for (int k = p.cta_begin[blockIdx.x]; k < k_end; ++k) {
-    const WorkItem w = load_item(p.items, k);
-    if (w.head[s] < 0) continue;
-    const int row = w.qtile[s] * kTile + r;
-    const size_t out_row = (size_t(w.batch) * p.heads_q + w.head[s]) * size_t(p.seq_q) + size_t(row);
+    const Item w = load_item(p.items, k);
+    if (w.head(s) < 0) continue;
+    const int row = w.qtile(s) * kTile + r;
+    const size_t out_row = (size_t(w.batch) * p.heads_q + w.head(s)) * size_t(p.seq_q) + size_t(row);
     float m_ref = -CUDART_INF_F, l = 0.0f;
-    const bool active = w.hi[s] >= w.lo[s];
+    const int lo = w.lo(s), hi = w.hi(s);
+    const bool active = hi >= lo;
 
-    for (int t = w.lo[s]; t <= w.hi[s]; ++t) {
+    for (int t = lo; t <= hi; ++t) {
       // which key tile, and does it need the element-wise mask (case iii)?
       int j;
       bool partial;
       uint32_t sub = 0xF;
       if (w.kind == 0) {
         j = w.j0 + t;
-        const int i0 = w.qtile[s] * kTile, i1 = min(i0 + kTile - 1, p.seq_q - 1);
+        const int i0 = w.qtile(s) * kTile, i1 = min(i0 + kTile - 1, p.seq_q - 1);
         const int j0 = j * kTile, j1 = min(j0 + kTile - 1, p.seq_kv - 1);
         const bool full = (!causal || j1 <= i0 + off) && (!windowed || (i1 + off) - j0 < p.window) &&
                           (j1 - j0 + 1 == kTile);
         partial = !full;
       } else {
-        const StepPair sp = p.steps[w.list_off + t];
-        const uint32_t e = sp.e[s];
+        const uint2 sp = __ldg(reinterpret_cast<const uint2 *>(p.steps + w.list_off + t));
+        const uint32_t e = s ? sp.y : sp.x;
         j = int(e & kEntryTileMask);
         partial = (e & kEntryPartial) != 0;
         sub = (e >> kEntrySubShift) & 0xF;
       }
 
-      bool ok = bounded_wait(&ctrl.s_full[s], n_sp & 1u, ctrl, p.status);
-      ok = __all_sync(0xffffffffu, ok);
+      bool ok;
+      {
+        TRACE_T0();
+        ok = bounded_wait(&ctrl.s_full[s], n_sp & 1u, ctrl, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        TRACE_ADD(0);
+      }
       if (!ok) return;
-      ++n_sp;
       tc_fence_after();
+      TRACE_T0();
 
       float x[kTile];
 #pragma unroll
@@ -315,6 +461,7 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         for (int i = 0; i < 32; ++i) x[c * 32 + i] = __uint_as_float(regs[i]);
       }
       tc_wait_ld();
+      TRACE_ADD(2);
 
       if (partial) {
         // visible columns of this row form one interval [c_lo, c_hi] of the tile
@@ -329,17 +476,20 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         for (int c = 0; c < kTile; ++c) x[c] = (c >= c_lo && c <= c_hi) ? x[c] : -CUDART_INF_F;
       }
 
-      float mx0 = x[0], mx1 = x[1], mx2 = x[2], mx3 = x[3];
+      float mx0 = fmax3(x[0], x[1], x[2]), mx1 = fmax3(x[3], x[4], x[5]);
+      float mx2 = fmax3(x[6], x[7], x[8]), mx3 = fmax3(x[9], x[10], x[11]);
 #pragma unroll
-      for (int c = 4; c < kTile; c += 4) {
-        mx0 = fmaxf(mx0, x[c]);
-        mx1 = fmaxf(mx1, x[c + 1]);
-        mx2 = fmaxf(mx2, x[c + 2]);
-        mx3 = fmaxf(mx3, x[c + 3]);
+      for (int c = 12; c < 124; c += 8) {
+        mx0 = fmax3(mx0, x[c], x[c + 1]);
+        mx1 = fmax3(mx1, x[c + 2], x[c + 3]);
+        mx2 = fmax3(mx2, x[c + 4], x[c + 5]);
+        mx3 = fmax3(mx3, x[c + 6], x[c + 7]);
       }
+      mx0 = fmax3(mx0, x[124], x[125]);
+      mx1 = fmax3(mx1, x[126], x[127]);
       const float ms = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale_log2;
 
-      if (t == w.lo[s]) {
+      if (t == lo) {
         m_ref = ms;
       } else {
         // the running maximum only has to bound the exponents: rescale O lazily
@@ -360,40 +510,38 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         }
       }
       const float m_use = (m_ref == -CUDART_INF_F) ? 0.0f : m_ref;
+      const float2 neg_m2 = make_float2(-m_use, -m_use);
 
-      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      float2 acc_a = make_float2(0.f, 0.f), acc_b = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int half = 0; half < 2; ++half) {
         uint32_t packed[32];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const int e = c * 64 + 2 * i;
-          const float p0 = ex2_approx(fmaf(x[e], scale_log2, -m_use));
-          const float p1 = ex2_approx(fmaf(x[e + 1], scale_log2, -m_use));
-          const float p2 = ex2_approx(fmaf(x[e + 2], scale_log2, -m_use));
-          const float p3 = ex2_approx(fmaf(x[e + 3], scale_log2, -m_use));
-          l0 += p0;
-          l1 += p1;
-          l2 += p2;
-          l3 += p3;
-          packed[i] = pack_bf16x2(p0, p1);
-          packed[i + 1] = pack_bf16x2(p2, p3);
-        }
-        tmem_st32(t_s + c * 32, packed);
+        exp_half(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
+        tmem_st32(t_s + half * 32, packed);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl.p_full[s][half]);
       }
-      l += (l0 + l1) + (l2 + l3);
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(&ctrl.p_full[s]);
+      ++n_sp;
+      const float2 acc = fadd2(acc_a, acc_b);
+      l += acc.x + acc.y;
+      TRACE_ADD(3);
     }
 
     // epilogue: O / l and LSE = ln2 * (m + log2 l)
     if (active) {
-      bool ok = bounded_wait(&ctrl.o_full[s], n_use & 1u, ctrl, p.status);
-      ok = __all_sync(0xffffffffu, ok);
+      bool ok;
+      {
+        TRACE_T0();
+        ok = bounded_wait(&ctrl.o_full[s], n_use & 1u, ctrl, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        TRACE_ADD(1);
+      }
       if (!ok) return;
       ++n_use;
       tc_fence_after();
+      TRACE_T0();
       const float inv = l > 0.0f ? 1.0f / l : 0.0f;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -414,9 +562,11 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         }
       }
       tc_fence_before();
-      mbar_arrive(&ctrl.o_empty[s]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl.o_empty[s]);
       if (p.lse != nullptr && row < p.seq_q)
         p.lse[out_row] = l > 0.0f ? 0.6931471805599453f * (m_ref + log2f(l)) : -CUDART_INF_F;
+      TRACE_ADD(4);
     } else if (row < p.seq_q) {
       // no key tile is visible to this query tile
       uint4 *dst = reinterpret_cast<uint4 *>(o_base + out_row * D);
@@ -425,6 +575,12 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
       if (p.lse != nullptr) p.lse[out_row] = -CUDART_INF_F;
     }
   }
+#ifdef STEEL_TRACE
+  trace_acc[6] = clock64() - role_t0;
+  if (r == 0) {
+    TRACE_FLUSH(16 + 8 * s, 7);
+  }
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -449,10 +605,12 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(&ctrl.q_full[s], 1);
       mbar_init(&ctrl.q_empty[s], 1);
       mbar_init(&ctrl.s_full[s], 1);
-      mbar_init(&ctrl.p_full[s], kTile);
+      mbar_init(&ctrl.p_full[s][0], 4);  // one arrival per softmax warp
+      mbar_init(&ctrl.p_full[s][1], 4);
       mbar_init(&ctrl.o_full[s], 1);
-      mbar_init(&ctrl.o_empty[s], kTile);
+      mbar_init(&ctrl.o_empty[s], 4);
     }
+    for (int i = 0; i < kFifoDepth; ++i) ctrl.fifo[i] = 0;
     ctrl.abort = 0;
     fence_barrier_init();
   }
@@ -469,12 +627,19 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
 
-  if (warp < 8) {
-    softmax_role<D>(p, ctrl, warp / 4, threadIdx.x % kTile);
-  } else if (warp == kProducerWarp) {
-    if (lane == 0) producer_role<D>(p, &map_q, &map_k, &map_v, ctrl, smem_q, smem_ring);
+  if (warp < 4) {
+    setmaxnreg_inc<kRegsSoftmax>();
+    softmax_role<D, 0>(p, ctrl, threadIdx.x % kTile);
+  } else if (warp < 8) {
+    setmaxnreg_inc<kRegsSoftmax>();
+    softmax_role<D, 1>(p, ctrl, threadIdx.x % kTile);
   } else {
-    if (lane == 0) mma_role<D>(p, ctrl, smem_q, smem_ring);
+    setmaxnreg_dec<kRegsOther>();
+    if (warp == kProducerWarp) {
+      if (lane == 0) producer_role<D>(p, &map_q, &map_k, &map_v, ctrl, smem_q, smem_ring);
+    } else if (warp == kMmaWarp) {
+      if (lane == 0) mma_role<D>(p, ctrl, smem_q, smem_ring);
+    }
   }
 
   __syncwarp();

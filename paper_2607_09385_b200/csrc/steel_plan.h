@@ -52,6 +52,7 @@ struct KernelParams {
   uint32_t mask_flags;
   int32_t window;            // clamped to int32 range
   float scale_log2;          // scale * log2(e)
+  long long *trace;          // per-CTA wait accounting (debug builds only), else null
 };
 
 }  // namespace steel
