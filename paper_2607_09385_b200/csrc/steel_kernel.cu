@@ -34,6 +34,10 @@ constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr long long kTimeoutCycles = 4000000000ll;  // about two seconds
 constexpr float kRescaleThreshold = 8.0f;           // lazy rescale: P stays below 2^8
+#ifndef STEEL_EXP_EMULATION
+#define STEEL_EXP_EMULATION 0
+#endif
+constexpr int kExpEmulation = STEEL_EXP_EMULATION;  // 0 none, 1: 12.5 %, 2: 25 %, 3: 50 % of exp2 on the FMA pipe
 constexpr int kMaxStages = 10;
 constexpr int kFifoDepth = 32;
 constexpr uint32_t kMaskCausal = 1u, kMaskWindow = 2u;
@@ -93,6 +97,14 @@ __device__ __forceinline__ bool bounded_wait(uint64_t *bar, uint32_t parity, Ctr
       }
     }
   }
+}
+
+// One lane polls on behalf of its warp; the vote both broadcasts the outcome and orders the other
+// lanes after the observation.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, Ctrl &ctrl, int32_t *status, int lane) {
+  bool ok = true;
+  if (lane == 0) ok = bounded_wait(bar, parity, ctrl, status);
+  return __all_sync(0xffffffffu, ok);
 }
 
 // A work item unpacked into scalars (no indexable arrays, so everything stays in registers).
@@ -374,7 +386,27 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
 }
 
 // ------------------------------------------------------------------------------------------------
-// exp2 of 64 scaled scores -> 32 packed bf16x2 registers; accumulates the row sum in two lanes pairs.
+// 2^y for a pair of exponents on the FMA pipe instead of the special-function unit: y = n + f with
+// n = round(y), f in [-0.5, 0.5]; 2^f by a cubic with 7.5e-5 relative error (far below bf16's
+// 2^-9), scaled by adding n to the exponent field.  Inputs must be finite or -inf; they are clamped
+// at -125 so the exponent field stays positive (the result is then at most 2^-125).
+__device__ __forceinline__ float2 exp2_poly(float2 y) {
+  const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to the nearest integer
+  y.x = fmaxf(y.x, -125.0f);
+  y.y = fmaxf(y.y, -125.0f);
+  const float2 t = fadd2(y, make_float2(kMagic, kMagic));
+  const float2 f = fadd2(y, fadd2(make_float2(kMagic, kMagic), make_float2(-t.x, -t.y)));
+  float2 q = ffma2(make_float2(5.517166907e-02f, 5.517166907e-02f), f, make_float2(2.426111222e-01f, 2.426111222e-01f));
+  q = ffma2(q, f, make_float2(6.932609855e-01f, 6.932609855e-01f));
+  q = ffma2(q, f, make_float2(9.999280735e-01f, 9.999280735e-01f));
+  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
+  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
+  return q;
+}
+
+// exp2 of 64 scaled scores -> 32 packed bf16x2 registers; accumulates the row sum in two lane pairs.
+// With kEmu > 0, one pair in every 2^(3 - kEmu) is evaluated by exp2_poly (12.5 %, 25 %, 50 %).
+template <int kEmu>
 __device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, float2 scale2, float2 neg_m2,
                                          float2 &acc_a, float2 &acc_b, uint32_t (&packed)[32]) {
 #pragma unroll
@@ -384,8 +416,13 @@ __device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, floa
     float2 y1 = ffma2(make_float2(x[e + 2], x[e + 3]), scale2, neg_m2);
     y0.x = ex2_approx(y0.x);
     y0.y = ex2_approx(y0.y);
-    y1.x = ex2_approx(y1.x);
-    y1.y = ex2_approx(y1.y);
+    const bool emulate = kEmu > 0 && ((i / 2) % (1 << (3 - kEmu)) == (1 << (3 - kEmu)) - 1);
+    if (emulate) {
+      y1 = exp2_poly(y1);
+    } else {
+      y1.x = ex2_approx(y1.x);
+      y1.y = ex2_approx(y1.y);
+    }
     acc_a = fadd2(acc_a, y0);
     acc_b = fadd2(acc_b, y1);
     packed[i] = pack_bf16x2(y0.x, y0.y);
@@ -393,8 +430,8 @@ __device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, floa
   }
 }
 
-template <int D, int s>
-__device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int r) {
+template <int D>
+__device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, const int r) {
   using C = Cfg<D>;
   const int lane = r % 32;
   const uint32_t lane_base = uint32_t((r / 32) * 32) << 16;
@@ -444,8 +481,7 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int r) {
       bool ok;
       {
         TRACE_T0();
-        ok = bounded_wait(&ctrl.s_full[s], n_sp & 1u, ctrl, p.status);
-        ok = __all_sync(0xffffffffu, ok);
+        ok = warp_wait(&ctrl.s_full[s], n_sp & 1u, ctrl, p.status, lane);
         TRACE_ADD(0);
       }
       if (!ok) return;
@@ -516,7 +552,9 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int r) {
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t packed[32];
-        exp_half(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
+        // masked (-inf) scores keep the exact special-function path so that empty rows sum to 0
+        if (kExpEmulation == 0 || partial) exp_half<0>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
+        else exp_half<kExpEmulation>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
         tmem_st32(t_s + half * 32, packed);
         tc_wait_st();
         tc_fence_before();
@@ -534,8 +572,7 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int r) {
       bool ok;
       {
         TRACE_T0();
-        ok = bounded_wait(&ctrl.o_full[s], n_use & 1u, ctrl, p.status);
-        ok = __all_sync(0xffffffffu, ok);
+        ok = warp_wait(&ctrl.o_full[s], n_use & 1u, ctrl, p.status, lane);
         TRACE_ADD(1);
       }
       if (!ok) return;
@@ -627,12 +664,9 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
 
-  if (warp < 4) {
+  if (warp < 8) {
     setmaxnreg_inc<kRegsSoftmax>();
-    softmax_role<D, 0>(p, ctrl, threadIdx.x % kTile);
-  } else if (warp < 8) {
-    setmaxnreg_inc<kRegsSoftmax>();
-    softmax_role<D, 1>(p, ctrl, threadIdx.x % kTile);
+    softmax_role<D>(p, ctrl, warp / 4, threadIdx.x % kTile);
   } else {
     setmaxnreg_dec<kRegsOther>();
     if (warp == kProducerWarp) {
