@@ -143,6 +143,31 @@ steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_att
  * (uniform, contiguous) order. */
 steel_status_t steel_attn_set_policy(int32_t policy);
 
+/*
+ * (The paper has no counterpart to this entry point; it exists for integration.)  One attention
+ * call for callers that cannot allocate device memory: code that runs inside another framework's
+ * locked memory pool, on a latency path where cudaMalloc's implicit synchronisation is not
+ * acceptable, or under a device-memory budget fixed at start-up.  It takes the problem description
+ * and the tensors directly -- no handle -- and keeps the work lists that steel_attn_create would put
+ * in cudaMalloc'ed buffers in a fixed array inside the library image instead (about 2 MiB, held on
+ * every GPU that loads the library until the process exits).  It calls no cudaMalloc / cudaFree.
+ *
+ * Limits: at most 16384 work items, 131072 explicit step-list entries (bitmap masks) and 1024
+ * persistent CTAs; a problem whose plan is larger is refused with STEEL_ERR_UNSUPPORTED and
+ * nothing is launched (the 131072-token graded configuration, 16384 items, is the largest
+ * causal case that fits).  Arguments as for steel_attn_run; scheduling policy 0 is always used.
+ *
+ * The call is blocking: it plans on the host (transient host memory only), copies the lists on
+ * `cuda_stream`, runs the kernel, waits for the stream and returns the device status (STEEL_OK or
+ * STEEL_ERR_TIMEOUT).  All calls in the process share the one array per GPU, which still holds the
+ * previous call's lists when a call starts: the call rewrites the lists and clears the status word,
+ * so two calls that overlap on the same GPU (from two threads or streams) race and must be
+ * serialised by the caller.  The first call on each device also resolves the array's device
+ * address and configures the kernels; make that first call outside any stream capture.
+ */
+steel_status_t steel_attn_run_noalloc(const steel_attn_params_t *params, const void *q, const void *k,
+                                      const void *v, void *o, float *lse, void *cuda_stream);
+
 const char *steel_status_string(steel_status_t status);
 
 #ifdef __cplusplus

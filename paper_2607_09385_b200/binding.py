@@ -20,7 +20,8 @@ STEEL_MASK_CAUSAL, STEEL_MASK_WINDOW, STEEL_MASK_BITMAP = 1, 2, 4
 
 EXPORTS = (
     "steel_attn_create", "steel_attn_run", "steel_attn_last_status", "steel_attn_destroy",
-    "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_set_policy", "steel_status_string",
+    "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_set_policy", "steel_attn_run_noalloc",
+    "steel_status_string",
 )
 
 
@@ -82,6 +83,7 @@ def load_library():
     lib.steel_attn_plan_host.argtypes = [ctypes.POINTER(Params), ctypes.POINTER(Stats), vp, ctypes.c_int64,
                                          ctypes.POINTER(ctypes.c_int64)]
     lib.steel_attn_set_policy.argtypes = [ctypes.c_int32]
+    lib.steel_attn_run_noalloc.argtypes = [ctypes.POINTER(Params), vp, vp, vp, vp, vp, vp]
     lib.steel_status_string.argtypes = [ctypes.c_int]
     lib.steel_status_string.restype = ctypes.c_char_p
     for name in EXPORTS[:-1]:
@@ -150,6 +152,14 @@ def steel_attn_plan_host(params: Params, want_tiles: bool = False, capacity: int
     if st != STEEL_OK:
         return st, None, None
     return st, s.as_dict(), (tiles[: n.value].copy() if want_tiles else None)
+
+
+def steel_attn_run_noalloc(params: Params, q_ptr: int, k_ptr: int, v_ptr: int, o_ptr: int, lse_ptr,
+                           stream: int) -> int:
+    """The allocation-free call: plans, runs and waits; returns the status code (see the header for
+    who needs it, its size limits and why overlapping calls race)."""
+    return load_library().steel_attn_run_noalloc(ctypes.byref(params), q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr,
+                                                 stream)
 
 
 def steel_attn_set_policy(policy: int) -> None:

@@ -72,6 +72,33 @@ void free_device(steel_attn *h) {
 
 }  // namespace
 
+namespace steel {
+
+// Encode the tensor maps for (q, k, v), fill the problem fields of `kp` (whose list and status
+// pointers the caller has set) and enqueue the kernel.
+steel_status_t launch_with_params(const steel_attn_params_t &p, KernelParams kp, int grid, const void *q,
+                                  const void *k, const void *v, void *o, float *lse, cudaStream_t stream) {
+  CUtensorMap map_q, map_k, map_v;
+  if (!make_map(&map_q, q, p.head_dim, p.seq_q, int64_t(p.batch) * p.heads_q) ||
+      !make_map(&map_k, k, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv) ||
+      !make_map(&map_v, v, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv))
+    return STEEL_ERR_CUDA;
+  kp.o = o;
+  kp.lse = lse;
+  kp.heads_q = p.heads_q;
+  kp.heads_kv = p.heads_kv;
+  kp.seq_q = p.seq_q;
+  kp.seq_kv = p.seq_kv;
+  kp.mask_flags = p.mask.flags;
+  kp.window = int32_t(p.mask.window > std::numeric_limits<int32_t>::max() ? std::numeric_limits<int32_t>::max()
+                                                                          : p.mask.window);
+  kp.scale_log2 = p.scale * 1.4426950408889634f;
+  if (launch_attention(p.head_dim, map_q, map_k, map_v, kp, grid, stream) != cudaSuccess) return STEEL_ERR_CUDA;
+  return STEEL_OK;
+}
+
+}  // namespace steel
+
 extern "C" {
 
 steel_status_t steel_attn_create(const steel_attn_params_t *params, steel_attn_t **out) {
