@@ -33,7 +33,7 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one kernel launch on the default workload,
 # from the ncu capture summarised in profiles/ (None until a capture exists for a workload).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"c4_bitmap25_s32k_h16": 4 * (140.947968e6 + 15.088640e6)}  # 4 x the 4-head capture
 
 
 def load_peaks():
@@ -118,6 +118,14 @@ def time_oracle(w, data, n_rows: int, effective_flop: float):
     return effective_flop * share / dt / 1e12, dt, oracle.max_threads()
 
 
+def calibrate_rows(w, data, effective_flop: float, target_seconds: float, cap: int = 1 << 17) -> int:
+    """Number of sampled rows that makes one oracle pass last about `target_seconds` on this host."""
+    probe = 128
+    _, dt, _ = time_oracle(w, data, probe, effective_flop)
+    rows = int(probe * target_seconds / max(dt, 1e-4))
+    return max(probe, min(rows, cap, w.batch * w.heads_q * w.seq))
+
+
 def plan_stats(w, bitmap):
     from paper_2607_09385_b200 import binding
     params, _keep = binding.make_params(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim, w.scale,
@@ -133,7 +141,9 @@ def run_reference(args, w, rank, world):
         return
     data = inputs.make_inputs(w, inputs.DEFAULT_SEED)
     stats = plan_stats(w, data["bitmap"])
-    n_rows = args.oracle_rows
+    # a bounded sample per step: the whole run (warm-up + steps) aims at about a minute of oracle time
+    n_rows = args.oracle_rows or calibrate_rows(w, data, stats["effective_flop"],
+                                                60.0 / max(1, args.steps + args.warmup / 8.0))
     for _ in range(args.warmup):
         time_oracle(w, data, max(8, n_rows // 8), stats["effective_flop"])
     vals, secs = [], []
@@ -163,7 +173,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=25)
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--impl", default="steel", choices=["steel", "reference"])
-    ap.add_argument("--oracle-rows", type=int, default=1024)
+    ap.add_argument("--oracle-rows", type=int, default=0,
+                    help="rows the CPU oracle is timed on (0: calibrated to about 12 s of wall time)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--policy", type=int, default=0)
@@ -285,9 +296,10 @@ def main():
                     "hbm_min_bytes": 2 * (q.numel() * 2) + 2 * (k.numel() * 2) + lse.numel() * 4}
         cpu = None
         if not args.no_cpu_baseline:
-            val, dt, threads = time_oracle(w, data, args.oracle_rows, flop)
+            n_rows = args.oracle_rows or calibrate_rows(w, data, flop, 12.0)
+            val, dt, threads = time_oracle(w, data, n_rows, flop)
             cpu = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
-                   "sample": f"{args.oracle_rows} seeded random query rows of {w.name} "
+                   "sample": f"{n_rows} seeded random query rows of {w.name} "
                              f"(dense fp64 rows over all {w.seq} keys), scaled by rows/total rows"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
