@@ -65,7 +65,7 @@ struct Ctrl {
 constexpr uint32_t kCmdValid = 1u << 0, kCmdIsS = 1u << 1, kCmdSlot1 = 1u << 2, kCmdRingShift = 3,  // 4 bits
                    kCmdRingPhase = 1u << 7, kCmdWaitFirst = 1u << 8, kCmdFirstPhase = 1u << 9,
                    kCmdFinalUse = 1u << 10, kCmdEnd = 1u << 11, kCmdAcc = 1u << 12, kCmdPPhase = 1u << 13,
-                   kCmdExit = 1u << 14;
+                   kCmdExit = 1u << 14, kCmdSkipRingWait = 1u << 15;
 
 // Optional per-role wait accounting (compiled in with -DSTEEL_TRACE only): cycles per CTA, 32 slots.
 #ifdef STEEL_TRACE
@@ -286,8 +286,9 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
       }
       // phase of this item's use of the slot: Q-full for S, O-empty (inverted) for PV
       const uint32_t use_phase = ((s ? n_use1 : n_use0) - 1u) & 1u;
+      // the second user of a shared fill is issued after the first, which already waited for the load
       uint32_t cmd = kCmdValid | (f.slot << kCmdRingShift) | (f.phase ? kCmdRingPhase : 0u) |
-                     (s ? kCmdSlot1 : 0u) | (final_use ? kCmdFinalUse : 0u);
+                     (s ? kCmdSlot1 : 0u) | (final_use ? kCmdFinalUse : 0u) | (first ? 0u : kCmdSkipRingWait);
       if (t == w.lo(s)) cmd |= kCmdWaitFirst;
       if (t == w.hi(s)) cmd |= kCmdEnd;
       if (is_s) {
@@ -341,15 +342,17 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
   const uint64_t desc_k0 = make_smem_desc(smem_u32(smem_ring), 16, 1024);
   const uint64_t desc_v0 = make_smem_desc(smem_u32(smem_ring), C::kBoxBytes, 1024);
   uint32_t head = 0;
-  while (true) {
-    const uint32_t cmd = fifo_pop(ctrl, head, p.status);
-    if (cmd & kCmdExit) break;
+  uint32_t cmd = fifo_pop(ctrl, head, p.status);
+  while (!(cmd & kCmdExit)) {
+    // look at the next command now, so that its shared-memory latency hides behind this one's issue
+    volatile uint32_t *next_cell = &ctrl.fifo[head];
+    const uint32_t next = *next_cell;
     const uint32_t s = (cmd & kCmdSlot1) ? 1u : 0u;
     const uint32_t slot = (cmd >> kCmdRingShift) & 0xFu, ring_phase = (cmd & kCmdRingPhase) ? 1u : 0u;
     const uint32_t first_phase = (cmd & kCmdFirstPhase) ? 1u : 0u;
     if (cmd & kCmdIsS) {
       if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.q_full[s], first_phase, ctrl, p.status)) break;
-      if (!bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
+      if (!(cmd & kCmdSkipRingWait) && !bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
       tc_fence_after();
       const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
       const uint64_t dk = desc_k0 + uint64_t((slot * C::kTileBytes) >> 4);
@@ -364,7 +367,7 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
       if (cmd & kCmdEnd) tc_commit(&ctrl.q_empty[s]);
     } else {
       if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.o_empty[s], first_phase, ctrl, p.status)) break;
-      if (!bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
+      if (!(cmd & kCmdSkipRingWait) && !bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
       const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
       const uint32_t t_o = tmem + C::kColO + s * D, t_p = tmem + C::kColS + s * kTile;
       const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u, p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
@@ -381,6 +384,13 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
       if (!ok) break;
       if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
       if (cmd & kCmdEnd) tc_commit(&ctrl.o_full[s]);
+    }
+    if (next != 0) {
+      *next_cell = 0;
+      head = (head + 1) & (kFifoDepth - 1);
+      cmd = next;
+    } else {
+      cmd = fifo_pop(ctrl, head, p.status);
     }
   }
 }
