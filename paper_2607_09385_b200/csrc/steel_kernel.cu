@@ -5,8 +5,7 @@
 //   warps 0-3 / 4-7 : softmax warpgroup of slot 0 / 1.  Thread r owns query row r: it reads the
 //                     score row S (fp32) from TMEM, applies scale and (partial tiles only) the mask
 //                     computed from coordinates, keeps the running maximum m and sum l, writes
-//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S (in two halves, so the
-//                     second product can start on the first), rescales O when the maximum has grown,
+//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S, rescales O when the maximum has grown,
 //                     and at the end writes O / l and LSE.  (Algorithm 1: scale_and_mask and rowmax of
 //                     the First Stage, the Second Stage, and the rescale of the Third.)
 //   warp 8          : TMA producer.  Loads Q once per item and K_j / V_j for executed tiles only into
@@ -55,7 +54,7 @@ struct Cfg {
 
 struct Ctrl {
   uint64_t ring_full[kMaxStages], ring_empty[kMaxStages];
-  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2][2], o_full[2], o_empty[2];
+  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2], o_empty[2];
   uint32_t fifo[kFifoDepth];  // command words from the producer to the MMA issuer (0 = empty)
   uint32_t tmem_base;
   int abort;
@@ -371,17 +370,11 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
       const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
       const uint32_t t_o = tmem + C::kColO + s * D, t_p = tmem + C::kColS + s * kTile;
       const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u, p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
-      bool ok = true;
+      if (!bounded_wait(&ctrl.p_full[s], p_phase, ctrl, p.status)) break;
+      tc_fence_after();
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        ok = bounded_wait(&ctrl.p_full[s][half], p_phase, ctrl, p.status);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-          mma_ts(t_o, t_p + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
-      }
-      if (!ok) break;
+      for (int kk = 0; kk < kTile / 16; ++kk)
+        mma_ts(t_o, t_p + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
       if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
       if (cmd & kCmdEnd) tc_commit(&ctrl.o_full[s]);
     }
@@ -566,11 +559,11 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         if (kExpEmulation == 0 || partial) exp_half<0>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
         else exp_half<kExpEmulation>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
         tmem_st32(t_s + half * 32, packed);
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ctrl.p_full[s][half]);
       }
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl.p_full[s]);
       ++n_sp;
       const float2 acc = fadd2(acc_a, acc_b);
       l += acc.x + acc.y;
@@ -652,8 +645,7 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(&ctrl.q_full[s], 1);
       mbar_init(&ctrl.q_empty[s], 1);
       mbar_init(&ctrl.s_full[s], 1);
-      mbar_init(&ctrl.p_full[s][0], 4);  // one arrival per softmax warp
-      mbar_init(&ctrl.p_full[s][1], 4);
+      mbar_init(&ctrl.p_full[s], 4);  // one arrival per softmax warp
       mbar_init(&ctrl.o_full[s], 1);
       mbar_init(&ctrl.o_empty[s], 4);
     }
