@@ -139,8 +139,10 @@ steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_att
 /* Number of scheduler policies and selection of one for subsequently created handles
  * (process-wide; default 0).  0: query tiles paired for shared K/V loads, items ordered
  * KV-head-major then longest first (the sparsity-aware placement idea of the paper's Sec.
- * "Sparsity-Aware Pipeline Placement" recast for persistent CTAs); 1: same items in natural
- * (uniform, contiguous) order. */
+ * "Sparsity-Aware Pipeline Placement" recast for persistent CTAs); 1: the same items in natural
+ * order cut into contiguous chunks, one per CTA (the paper's "uniform placement"); 2: the same
+ * items dealt round-robin to the CTAs (the paper's sparsity-aware placement: consecutive query
+ * tiles side by side). */
 steel_status_t steel_attn_set_policy(int32_t policy);
 
 /*

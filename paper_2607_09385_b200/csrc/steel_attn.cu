@@ -259,7 +259,7 @@ steel_status_t steel_attn_set_trace(steel_attn_t *h, long long *device_buffer) {
 #endif
 
 steel_status_t steel_attn_set_policy(int32_t policy) {
-  if (policy < 0 || policy > 1) return STEEL_ERR_INVALID_ARG;
+  if (policy < 0 || policy > 2) return STEEL_ERR_INVALID_ARG;
   g_policy.store(policy);
   return STEEL_OK;
 }

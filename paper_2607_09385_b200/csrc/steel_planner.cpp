@@ -359,11 +359,19 @@ steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy
       load[sl.second] = sl.first;
       heap.push(sl);
     }
-  } else {
+  } else if (policy == 1) {
     // uniform placement: contiguous chunks of the natural order
     size_t n = order.size();
     for (size_t k = 0; k < n; ++k) {
       int cta = int(k * size_t(grid) / std::max<size_t>(n, 1));
+      per_cta[cta].push_back(order[k]);
+      load[cta] += drafts[order[k]].w.n_steps + kItemOverheadSteps;
+    }
+  } else {
+    // interleaved placement: consecutive items of the natural order go to consecutive CTAs, so
+    // that CTAs working side by side hold query tiles of similar sparsity
+    for (size_t k = 0; k < order.size(); ++k) {
+      int cta = int(k % size_t(grid));
       per_cta[cta].push_back(order[k]);
       load[cta] += drafts[order[k]].w.n_steps + kItemOverheadSteps;
     }

@@ -145,12 +145,13 @@ def test_determinism_and_handle_reuse():
     attn.close()
 
 
-def test_uniform_policy_matches():
-    """The uniform (contiguous) placement computes the same result as the default placement."""
+@pytest.mark.parametrize("policy", [1, 2])
+def test_other_placement_policies_match(policy):
+    """Uniform (contiguous) and interleaved placement compute the same result as the default."""
     w = inputs.Workload("policy", 1, 4, 4, 2048, 128, 128, CAUSAL)
     data = inputs.make_inputs(w, seed=31)
     attn0, o0, lse0 = H.run_gpu(w, data)
-    binding.steel_attn_set_policy(1)
+    binding.steel_attn_set_policy(policy)
     try:
         attn1, o1, lse1 = H.run_gpu(w, data)
     finally:

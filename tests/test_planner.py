@@ -147,14 +147,20 @@ def test_balance_and_policies():
     stats, recs0 = host_plan(1, w.heads_q, w.heads_kv, w.seq, w.seq, 128, w.flags, tiles=True)
     assert stats["grid"] == 148
     assert stats["max_cta_steps"] <= 1.08 * stats["steps"] / 148 + 2
-    B.steel_attn_set_policy(1)
-    try:
-        stats1, recs1 = host_plan(1, w.heads_q, w.heads_kv, w.seq, w.seq, 128, w.flags, tiles=True)
-    finally:
-        B.steel_attn_set_policy(0)
     key = lambda r: {tuple(x[1:5]) for x in r}
-    assert key(recs0) == key(recs1) and stats1["exec_tiles"] == stats["exec_tiles"]
-    assert stats1["max_cta_steps"] > stats["max_cta_steps"]   # contiguous chunks are unbalanced under causal
+    by_policy = {0: stats}
+    for policy in (1, 2):
+        B.steel_attn_set_policy(policy)
+        try:
+            by_policy[policy], recs = host_plan(1, w.heads_q, w.heads_kv, w.seq, w.seq, 128, w.flags, tiles=True)
+        finally:
+            B.steel_attn_set_policy(0)
+        assert key(recs0) == key(recs) and by_policy[policy]["exec_tiles"] == stats["exec_tiles"]
+    # contiguous chunks (uniform placement) are the most unbalanced under a causal mask, dealing
+    # consecutive tiles round-robin (sparsity-aware placement) is better, longest-first is best
+    assert by_policy[1]["max_cta_steps"] > by_policy[2]["max_cta_steps"] > by_policy[0]["max_cta_steps"]
+    lib = B.load_library()
+    assert lib.steel_attn_set_policy(3) == B.STEEL_ERR_INVALID_ARG
 
 
 def test_makespan_model_of_uniform_vs_interleaved_placement():
