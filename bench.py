@@ -166,6 +166,38 @@ def run_reference(args, w, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_paper_sweep(args, dev):
+    """Throughput against sequence length on the paper's own shapes (BERT and Llama-3.1-1B attention,
+    head_dim 64): one JSON line with one entry per shape."""
+    import torch
+    from paper_2607_09385_b200 import binding
+    rows = []
+    for w in inputs.paper_workloads():
+        data = inputs.make_inputs(w, inputs.DEFAULT_SEED)
+        attn = binding.SteelAttention(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim, w.scale, w.flags,
+                                      w.block, w.window, None)
+        q, k, v = (torch.from_numpy(data[x].view(np.int16)).to(dev).view(torch.bfloat16) for x in "qkv")
+        o = torch.empty_like(q)
+        lse = torch.empty((w.batch, w.heads_q, w.seq), dtype=torch.float32, device=dev)
+        for _ in range(max(3, args.warmup)):
+            attn.run(q, k, v, o, lse)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            attn.run(q, k, v, o, lse)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        flop = attn.stats()["effective_flop"]
+        rows.append({"workload": w.name, "seq": w.seq, "heads": w.heads_q, "head_dim": w.head_dim,
+                     "causal": bool(w.flags & inputs.MASK_CAUSAL), "ms_per_call": ms,
+                     "tflops": flop / (ms * 1e-3) / 1e12})
+        attn.close()
+    print(json.dumps({"sweep": "paper", "metric": METRIC, "unit": UNIT, "steps": args.steps, "results": rows}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -178,6 +210,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--policy", type=int, default=0)
+    ap.add_argument("--sweep", default="", choices=["", "paper"],
+                    help="'paper': time the paper's own attention shapes (head_dim 64) instead of one workload")
     ap.add_argument("--profile-heads", type=int, default=0,
                     help="shrink the workload to this many query heads (same KV grouping) for ncu captures")
     args = ap.parse_args()
@@ -208,6 +242,10 @@ def main():
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.sweep == "paper":
+        run_paper_sweep(args, dev)
+        return
 
     # every rank works on its own replica (independent problem, own seed)
     data = inputs.make_inputs(w, inputs.DEFAULT_SEED + rank)

@@ -145,10 +145,22 @@ WORKLOADS = (
 )
 
 
+def paper_workloads():
+    """Attention shapes the paper itself evaluates (head_dim 64): BERT (12 heads, bidirectional,
+    S = 512 ... 4096; Sec. "Comparison with State-of-the-Art on NPU") and Llama-3.1-1B (32 heads,
+    causal, S = 2048 ... 32768; Sec. "Attention Benchmark")."""
+    out = []
+    for s in (512, 1024, 2048, 4096):
+        out.append(Workload(f"bert_h12_d64_s{s}", 1, 12, 12, s, 64, 128, 0))
+    for s in (2048, 4096, 8192, 16384, 32768):
+        out.append(Workload(f"llama1b_h32_d64_s{s}", 1, 32, 32, s, 64, 128, MASK_CAUSAL))
+    return out
+
+
 def workload(name_or_index) -> Workload:
     if isinstance(name_or_index, int):
         return WORKLOADS[name_or_index]
-    for w in WORKLOADS:
+    for w in WORKLOADS + tuple(paper_workloads()):
         if w.name == name_or_index or w.name.split("_")[0] == name_or_index:
             return w
     raise KeyError(name_or_index)

@@ -92,6 +92,17 @@ def test_edge_cases_all_rows(case):
     attn.close()
 
 
+@pytest.mark.parametrize("name", ["bert_h12_d64_s512", "llama1b_h32_d64_s2048"])
+def test_paper_shapes_head_dim_64(name):
+    """The paper's own attention shapes (BERT bidirectional, Llama-3.1-1B causal; head_dim 64)."""
+    w = inputs.workload(name)
+    data = inputs.make_inputs(w, seed=64)
+    attn, o, lse = H.run_gpu(w, data)
+    rows = H.all_rows(w) if w.seq <= 512 else H.sampled_rows(w, range(0, w.heads_q, 3), 1, 512)
+    H.assert_parity(w, data, o, lse, rows)
+    attn.close()
+
+
 def test_seq_q_differs_from_seq_kv():
     """Bottom-right aligned causal mask with more keys than queries, and the reverse (rows with no
     visible key give O = 0, LSE = -inf)."""
