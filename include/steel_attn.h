@@ -136,6 +136,15 @@ steel_status_t steel_attn_get_stats(const steel_attn_t *handle, steel_attn_stats
 steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_attn_stats_t *stats,
                                     int32_t *tiles, int64_t capacity, int64_t *n_tiles);
 
+/*
+ * Test hook for the bounded device-side waits.  With cta >= 0, CTA `cta` of the handle's following
+ * runs withholds the commands its producer would publish, so the waits of its other roles expire
+ * after `timeout_cycles` SM cycles (<= 0: the default, about two seconds): the kernel then returns
+ * normally, outputs are undefined and steel_attn_last_status reports STEEL_ERR_TIMEOUT.  Nothing
+ * faults or hangs; the context stays usable.  cta < 0 switches the hook off.
+ */
+steel_status_t steel_attn_debug_stall(steel_attn_t *handle, int32_t cta, int64_t timeout_cycles);
+
 /* Number of scheduler policies and selection of one for subsequently created handles
  * (process-wide; default 0).  0: query tiles paired for shared K/V loads, items ordered
  * KV-head-major then longest first (the sparsity-aware placement idea of the paper's Sec.

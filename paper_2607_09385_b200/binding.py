@@ -21,6 +21,7 @@ STEEL_MASK_CAUSAL, STEEL_MASK_WINDOW, STEEL_MASK_BITMAP = 1, 2, 4
 EXPORTS = (
     "steel_attn_create", "steel_attn_run", "steel_attn_last_status", "steel_attn_destroy",
     "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_set_policy", "steel_attn_run_noalloc",
+    "steel_attn_debug_stall",
     "steel_status_string",
 )
 
@@ -83,6 +84,7 @@ def load_library():
     lib.steel_attn_plan_host.argtypes = [ctypes.POINTER(Params), ctypes.POINTER(Stats), vp, ctypes.c_int64,
                                          ctypes.POINTER(ctypes.c_int64)]
     lib.steel_attn_set_policy.argtypes = [ctypes.c_int32]
+    lib.steel_attn_debug_stall.argtypes = [vp, ctypes.c_int32, ctypes.c_int64]
     lib.steel_attn_run_noalloc.argtypes = [ctypes.POINTER(Params), vp, vp, vp, vp, vp, vp]
     lib.steel_status_string.argtypes = [ctypes.c_int]
     lib.steel_status_string.restype = ctypes.c_char_p
@@ -160,6 +162,12 @@ def steel_attn_run_noalloc(params: Params, q_ptr: int, k_ptr: int, v_ptr: int, o
     who needs it, its size limits and why overlapping calls race)."""
     return load_library().steel_attn_run_noalloc(ctypes.byref(params), q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr,
                                                  stream)
+
+
+def steel_attn_debug_stall(handle: int, cta: int, timeout_cycles: int = 0) -> None:
+    st = load_library().steel_attn_debug_stall(handle, cta, timeout_cycles)
+    if st != STEEL_OK:
+        raise SteelError(st, "steel_attn_debug_stall")
 
 
 def steel_attn_set_policy(policy: int) -> None:

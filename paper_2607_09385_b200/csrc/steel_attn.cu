@@ -23,6 +23,8 @@ struct steel_attn {
   StepPair *d_steps = nullptr;
   int32_t *d_status = nullptr;
   long long *d_trace = nullptr;  // debug builds only
+  long long timeout_cycles = kDefaultTimeoutCycles;
+  int32_t stall_cta = -1;
 };
 
 namespace {
@@ -187,6 +189,8 @@ steel_status_t steel_attn_run(steel_attn_t *h, const void *q, const void *k, con
                                                                           : p.mask.window);
   kp.scale_log2 = p.scale * 1.4426950408889634f;
   kp.trace = h->d_trace;
+  kp.timeout_cycles = h->timeout_cycles;
+  kp.stall_cta = h->stall_cta;
   if (launch_attention(p.head_dim, map_q, map_k, map_v, kp, h->grid, static_cast<cudaStream_t>(cuda_stream)) !=
       cudaSuccess)
     return STEEL_ERR_CUDA;
@@ -257,6 +261,13 @@ steel_status_t steel_attn_set_trace(steel_attn_t *h, long long *device_buffer) {
   return STEEL_OK;
 }
 #endif
+
+steel_status_t steel_attn_debug_stall(steel_attn_t *h, int32_t cta, int64_t timeout_cycles) {
+  if (!h || cta >= h->grid) return STEEL_ERR_INVALID_ARG;
+  h->stall_cta = cta < 0 ? -1 : cta;
+  h->timeout_cycles = timeout_cycles > 0 ? timeout_cycles : kDefaultTimeoutCycles;
+  return STEEL_OK;
+}
 
 steel_status_t steel_attn_set_policy(int32_t policy) {
   if (policy < 0 || policy > 2) return STEEL_ERR_INVALID_ARG;

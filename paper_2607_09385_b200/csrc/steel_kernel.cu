@@ -31,7 +31,6 @@ constexpr int kRegsSoftmax = 216;    // registers per thread after the warpgroup
 constexpr int kRegsOther = 72;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr long long kTimeoutCycles = 4000000000ll;  // about two seconds
 constexpr float kRescaleThreshold = 8.0f;           // lazy rescale: P stays below 2^8
 #ifndef STEEL_EXP_EMULATION
 #define STEEL_EXP_EMULATION 0
@@ -58,6 +57,7 @@ struct Ctrl {
   uint32_t fifo[kFifoDepth];  // command words from the producer to the MMA issuer (0 = empty)
   uint32_t tmem_base;
   int abort;
+  long long timeout_cycles;
 };
 
 // Command word layout (producer -> MMA issuer).
@@ -89,7 +89,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t *bar, uint32_t parity, Ctr
     if (mbar_try_wait(bar, parity)) return true;
     if ((++n & 63u) == 0) {
       if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return false;
-      if (clock64() - start > kTimeoutCycles) {
+      if (clock64() - start > ctrl.timeout_cycles) {
         *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
         atomicExch(status, 5);
         return false;
@@ -211,7 +211,7 @@ __device__ __forceinline__ bool fifo_push(Ctrl &ctrl, uint32_t &tail, uint32_t w
     while (*cell != 0) {
       if ((++n & 63u) == 0) {
         if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return false;
-        if (clock64() - start > kTimeoutCycles) {
+        if (clock64() - start > ctrl.timeout_cycles) {
           *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
           atomicExch(status, 5);
           return false;
@@ -232,7 +232,7 @@ __device__ __forceinline__ uint32_t fifo_pop(Ctrl &ctrl, uint32_t &head, int32_t
     while ((word = *cell) == 0) {
       if ((++n & 63u) == 0) {
         if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return kCmdExit;
-        if (clock64() - start > kTimeoutCycles) {
+        if (clock64() - start > ctrl.timeout_cycles) {
           *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
           atomicExch(status, 5);
           return kCmdExit;
@@ -254,6 +254,7 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
   RingPos ring{0, 0};
   uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, fills = 0, tail = 0;
   bool ok = true;
+  const bool stalled = p.stall_cta == int(blockIdx.x);
   const int k_end = p.cta_begin[blockIdx.x + 1];
   for (int k = p.cta_begin[blockIdx.x]; k < k_end && ok; ++k) {
     const Item w = load_item(p.items, k);
@@ -297,6 +298,7 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
         cmd |= ((use_phase ^ 1u) ? kCmdFirstPhase : 0u) | (t > w.lo(s) ? kCmdAcc : 0u) | ((n_sp & 1u) ? kCmdPPhase : 0u);
         ++n_sp;
       }
+      if (stalled) return true;  // test hook: the issuer's bounded wait for this command must expire
       return fifo_push(ctrl, tail, cmd, p.status);
     });
   }
@@ -313,7 +315,7 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
       }
       --slot;
       const long long start = clock64();
-      while (!mbar_try_wait(&ctrl.ring_full[slot], phase) && clock64() - start < kTimeoutCycles / 8) {
+      while (!mbar_try_wait(&ctrl.ring_full[slot], phase) && clock64() - start < ctrl.timeout_cycles / 8) {
       }
     }
 #pragma unroll
@@ -321,7 +323,7 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
       const uint32_t n_use = s ? n_use1 : n_use0;
       if (n_use) {
         const long long start = clock64();
-        while (!mbar_try_wait(&ctrl.q_full[s], (n_use - 1) & 1u) && clock64() - start < kTimeoutCycles / 8) {
+        while (!mbar_try_wait(&ctrl.q_full[s], (n_use - 1) & 1u) && clock64() - start < ctrl.timeout_cycles / 8) {
         }
       }
     }
@@ -651,6 +653,7 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     }
     for (int i = 0; i < kFifoDepth; ++i) ctrl.fifo[i] = 0;
     ctrl.abort = 0;
+    ctrl.timeout_cycles = p.timeout_cycles;
     fence_barrier_init();
   }
   if (warp == kProducerWarp && lane == 0) {

@@ -114,6 +114,8 @@ extern "C" steel_status_t steel_attn_run_noalloc(const steel_attn_params_t *para
   kp.steps = reinterpret_cast<const StepPair *>(base + kOffSteps);
   kp.status = reinterpret_cast<int32_t *>(base + kOffStatus);
   kp.trace = nullptr;
+  kp.timeout_cycles = kDefaultTimeoutCycles;
+  kp.stall_cta = -1;
   st = launch_with_params(*params, kp, plan.grid, q, k, v, o, lse, stream);
   if (st != STEEL_OK) return st;
   // Blocking by design: the host lists above must outlive the copies, and the status word has to

@@ -8,6 +8,7 @@
 namespace steel {
 
 constexpr int kTile = 128;  // query rows per tile and keys per tile
+constexpr long long kDefaultTimeoutCycles = 4000000000ll;  // about two seconds of SM clock
 
 // One step entry of one query tile ("slot") in a list-kind item.
 constexpr uint32_t kEntryTileMask = 0x00FFFFFFu;  // key-tile index
@@ -53,6 +54,8 @@ struct KernelParams {
   int32_t window;            // clamped to int32 range
   float scale_log2;          // scale * log2(e)
   long long *trace;          // per-CTA wait accounting (debug builds only), else null
+  long long timeout_cycles;  // bound of every device-side wait
+  int32_t stall_cta;         // test hook: this CTA's producer withholds its commands (-1: none)
 };
 
 }  // namespace steel
