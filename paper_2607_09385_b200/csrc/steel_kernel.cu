@@ -82,7 +82,7 @@ constexpr uint32_t kCmdValid = 1u << 0, kCmdIsS = 1u << 1, kCmdSlot1 = 1u << 2, 
 #endif
 
 __device__ __forceinline__ bool bounded_wait(uint64_t *bar, uint32_t parity, Ctrl &ctrl, int32_t *status) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_test_wait(bar, parity)) return true;  // the common case: already complete, no suspension
   const long long start = clock64();
   uint32_t n = 0;
   while (true) {
