@@ -60,11 +60,15 @@ struct Ctrl {
   long long timeout_cycles;
 };
 
-// Command word layout (producer -> MMA issuer).
-constexpr uint32_t kCmdValid = 1u << 0, kCmdIsS = 1u << 1, kCmdSlot1 = 1u << 2, kCmdRingShift = 3,  // 4 bits
-                   kCmdRingPhase = 1u << 7, kCmdWaitFirst = 1u << 8, kCmdFirstPhase = 1u << 9,
-                   kCmdFinalUse = 1u << 10, kCmdEnd = 1u << 11, kCmdAcc = 1u << 12, kCmdPPhase = 1u << 13,
-                   kCmdExit = 1u << 14, kCmdSkipRingWait = 1u << 15;
+// Command word (producer -> MMA issuer): one word carries PV(s, t), S(s, t + 1) or both (the usual
+// case: the second product of a step is followed at once by the first product of the next step).
+constexpr uint32_t kCmdValid = 1u << 0, kCmdHasPV = 1u << 1, kCmdHasS = 1u << 2, kCmdSlot1 = 1u << 3,
+                   kCmdVRingShift = 4, kCmdKRingShift = 8,  // 4 bits each: ring slot of the V / K tile
+                   kCmdVPhase = 1u << 12, kCmdKPhase = 1u << 13, kCmdVSkipWait = 1u << 14, kCmdKSkipWait = 1u << 15,
+                   kCmdVFinal = 1u << 16, kCmdKFinal = 1u << 17,  // last user: release the ring slot
+                   kCmdWaitOEmpty = 1u << 18, kCmdOEmptyPhase = 1u << 19, kCmdWaitQFull = 1u << 20,
+                   kCmdQFullPhase = 1u << 21, kCmdAcc = 1u << 22, kCmdPPhase = 1u << 23, kCmdOEnd = 1u << 24,
+                   kCmdQEnd = 1u << 25, kCmdExit = 1u << 31;
 
 // Optional per-role wait accounting (compiled in with -DSTEEL_TRACE only): cycles per CTA, 32 slots.
 #ifdef STEEL_TRACE
@@ -252,7 +256,7 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
                               const CUtensorMap *map_v, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring) {
   using C = Cfg<D>;
   RingPos ring{0, 0};
-  uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, fills = 0, tail = 0;
+  uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, fills = 0, tail = 0, pending = 0;
   bool ok = true;
   const bool stalled = p.stall_cta == int(blockIdx.x);
   const int k_end = p.cta_begin[blockIdx.x + 1];
@@ -286,20 +290,32 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
       }
       // phase of this item's use of the slot: Q-full for S, O-empty (inverted) for PV
       const uint32_t use_phase = ((s ? n_use1 : n_use0) - 1u) & 1u;
-      // the second user of a shared fill is issued after the first, which already waited for the load
-      uint32_t cmd = kCmdValid | (f.slot << kCmdRingShift) | (f.phase ? kCmdRingPhase : 0u) |
-                     (s ? kCmdSlot1 : 0u) | (final_use ? kCmdFinalUse : 0u) | (first ? 0u : kCmdSkipRingWait);
-      if (t == w.lo(s)) cmd |= kCmdWaitFirst;
-      if (t == w.hi(s)) cmd |= kCmdEnd;
       if (is_s) {
-        cmd |= kCmdIsS | (use_phase ? kCmdFirstPhase : 0u);
-      } else {
-        uint32_t &n_sp = s ? n_sp1 : n_sp0;
-        cmd |= ((use_phase ^ 1u) ? kCmdFirstPhase : 0u) | (t > w.lo(s) ? kCmdAcc : 0u) | ((n_sp & 1u) ? kCmdPPhase : 0u);
-        ++n_sp;
+        uint32_t part = kCmdHasS | (f.slot << kCmdKRingShift) | (f.phase ? kCmdKPhase : 0u) |
+                        (first ? 0u : kCmdKSkipWait) | (final_use ? kCmdKFinal : 0u);
+        if (t == w.lo(s)) part |= kCmdWaitQFull | (use_phase ? kCmdQFullPhase : 0u);
+        if (t == w.hi(s)) part |= kCmdQEnd;
+        // S(s, t) directly follows PV(s, t - 1) of the same slot: complete that command; otherwise
+        // (first step of the slot) it goes out alone
+        uint32_t cmd = pending | part | kCmdValid | (s ? kCmdSlot1 : 0u);
+        pending = 0;
+        if (stalled) return true;  // test hook: the issuer's bounded wait for this command must expire
+        return fifo_push(ctrl, tail, cmd, p.status);
       }
-      if (stalled) return true;  // test hook: the issuer's bounded wait for this command must expire
-      return fifo_push(ctrl, tail, cmd, p.status);
+      uint32_t &n_sp = s ? n_sp1 : n_sp0;
+      uint32_t part = kCmdHasPV | (f.slot << kCmdVRingShift) | (f.phase ? kCmdVPhase : 0u) |
+                      (first ? 0u : kCmdVSkipWait) | (final_use ? kCmdVFinal : 0u) | (t > w.lo(s) ? kCmdAcc : 0u) |
+                      ((n_sp & 1u) ? kCmdPPhase : 0u);
+      if (t == w.lo(s)) part |= kCmdWaitOEmpty | ((use_phase ^ 1u) ? kCmdOEmptyPhase : 0u);
+      ++n_sp;
+      if (t == w.hi(s)) {
+        // last step of the slot: no S follows
+        const uint32_t cmd = part | kCmdOEnd | kCmdValid | (s ? kCmdSlot1 : 0u);
+        if (stalled) return true;
+        return fifo_push(ctrl, tail, cmd, p.status);
+      }
+      pending = part;  // completed by the S(s, t + 1) that the walk visits next
+      return true;
     });
   }
   if (ok) ok = fifo_push(ctrl, tail, kCmdValid | kCmdExit, p.status);
@@ -349,36 +365,47 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
     volatile uint32_t *next_cell = &ctrl.fifo[head];
     const uint32_t next = *next_cell;
     const uint32_t s = (cmd & kCmdSlot1) ? 1u : 0u;
-    const uint32_t slot = (cmd >> kCmdRingShift) & 0xFu, ring_phase = (cmd & kCmdRingPhase) ? 1u : 0u;
-    const uint32_t first_phase = (cmd & kCmdFirstPhase) ? 1u : 0u;
-    if (cmd & kCmdIsS) {
-      if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.q_full[s], first_phase, ctrl, p.status)) break;
-      if (!(cmd & kCmdSkipRingWait) && !bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
+    const uint32_t t_s = tmem + C::kColS + s * kTile;
+    if (cmd & kCmdHasPV) {
+      const uint32_t slot = (cmd >> kCmdVRingShift) & 0xFu;
+      if ((cmd & kCmdWaitOEmpty) &&
+          !bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status))
+        break;
+      if (!(cmd & kCmdVSkipWait) &&
+          !bounded_wait(&ctrl.ring_full[slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status))
+        break;
+      if (!bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status)) break;
       tc_fence_after();
+      const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
+      const uint32_t t_o = tmem + C::kColO + s * D;
+      const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u;
+#pragma unroll
+      for (int kk = 0; kk < kTile / 16; ++kk)
+        mma_ts(t_o, t_s + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+      if (cmd & kCmdVFinal) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdOEnd) tc_commit(&ctrl.o_full[s]);
+    }
+    if (cmd & kCmdHasS) {
+      const uint32_t slot = (cmd >> kCmdKRingShift) & 0xFu;
+      if ((cmd & kCmdWaitQFull) &&
+          !bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status))
+        break;
+      if (!(cmd & kCmdKSkipWait) &&
+          !bounded_wait(&ctrl.ring_full[slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status))
+        break;
+      // after a PV of the same command the fence above still orders this product behind the
+      // softmax warps' reads of S
+      if (!(cmd & kCmdHasPV)) tc_fence_after();
       const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
       const uint64_t dk = desc_k0 + uint64_t((slot * C::kTileBytes) >> 4);
-      const uint32_t t_s = tmem + C::kColS + s * kTile;
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
         const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
         mma_ss(t_s, dq + off, dk + off, idesc_s, kk > 0);
       }
       tc_commit(&ctrl.s_full[s]);
-      if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
-      if (cmd & kCmdEnd) tc_commit(&ctrl.q_empty[s]);
-    } else {
-      if ((cmd & kCmdWaitFirst) && !bounded_wait(&ctrl.o_empty[s], first_phase, ctrl, p.status)) break;
-      if (!(cmd & kCmdSkipRingWait) && !bounded_wait(&ctrl.ring_full[slot], ring_phase, ctrl, p.status)) break;
-      const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
-      const uint32_t t_o = tmem + C::kColO + s * D, t_p = tmem + C::kColS + s * kTile;
-      const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u, p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
-      if (!bounded_wait(&ctrl.p_full[s], p_phase, ctrl, p.status)) break;
-      tc_fence_after();
-#pragma unroll
-      for (int kk = 0; kk < kTile / 16; ++kk)
-        mma_ts(t_o, t_p + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
-      if (cmd & kCmdFinalUse) tc_commit(&ctrl.ring_empty[slot]);
-      if (cmd & kCmdEnd) tc_commit(&ctrl.o_full[s]);
+      if (cmd & kCmdKFinal) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdQEnd) tc_commit(&ctrl.q_empty[s]);
     }
     if (next != 0) {
       *next_cell = 0;
