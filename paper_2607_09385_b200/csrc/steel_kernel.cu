@@ -366,45 +366,47 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
     const uint32_t next = *next_cell;
     const uint32_t s = (cmd & kCmdSlot1) ? 1u : 0u;
     const uint32_t t_s = tmem + C::kColS + s * kTile;
-    if (cmd & kCmdHasPV) {
-      const uint32_t slot = (cmd >> kCmdVRingShift) & 0xFu;
+    const uint32_t v_slot = (cmd >> kCmdVRingShift) & 0xFu, k_slot = (cmd >> kCmdKRingShift) & 0xFu;
+    const bool has_pv = (cmd & kCmdHasPV) != 0, has_s = (cmd & kCmdHasS) != 0;
+    // test the barriers this command depends on back to back, so their latencies overlap; only the
+    // ones not yet complete are then waited for
+    const bool need_v = has_pv && !(cmd & kCmdVSkipWait), need_k = has_s && !(cmd & kCmdKSkipWait);
+    bool ok_v = !need_v || mbar_test_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u);
+    bool ok_k = !need_k || mbar_test_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u);
+    bool ok_p = !has_pv || mbar_test_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u);
+    if (has_pv) {
       if ((cmd & kCmdWaitOEmpty) &&
           !bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status))
         break;
-      if (!(cmd & kCmdVSkipWait) &&
-          !bounded_wait(&ctrl.ring_full[slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status))
-        break;
-      if (!bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status)) break;
+      if (!ok_v && !bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status)) break;
+      if (!ok_p && !bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status)) break;
       tc_fence_after();
-      const uint64_t dv = desc_v0 + uint64_t((slot * C::kTileBytes) >> 4);
+      const uint64_t dv = desc_v0 + uint64_t((v_slot * C::kTileBytes) >> 4);
       const uint32_t t_o = tmem + C::kColO + s * D;
       const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u;
 #pragma unroll
       for (int kk = 0; kk < kTile / 16; ++kk)
         mma_ts(t_o, t_s + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
-      if (cmd & kCmdVFinal) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdVFinal) tc_commit(&ctrl.ring_empty[v_slot]);
       if (cmd & kCmdOEnd) tc_commit(&ctrl.o_full[s]);
     }
-    if (cmd & kCmdHasS) {
-      const uint32_t slot = (cmd >> kCmdKRingShift) & 0xFu;
+    if (has_s) {
       if ((cmd & kCmdWaitQFull) &&
           !bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status))
         break;
-      if (!(cmd & kCmdKSkipWait) &&
-          !bounded_wait(&ctrl.ring_full[slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status))
-        break;
+      if (!ok_k && !bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status)) break;
       // after a PV of the same command the fence above still orders this product behind the
       // softmax warps' reads of S
-      if (!(cmd & kCmdHasPV)) tc_fence_after();
+      if (!has_pv) tc_fence_after();
       const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
-      const uint64_t dk = desc_k0 + uint64_t((slot * C::kTileBytes) >> 4);
+      const uint64_t dk = desc_k0 + uint64_t((k_slot * C::kTileBytes) >> 4);
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
         const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
         mma_ss(t_s, dq + off, dk + off, idesc_s, kk > 0);
       }
       tc_commit(&ctrl.s_full[s]);
-      if (cmd & kCmdKFinal) tc_commit(&ctrl.ring_empty[slot]);
+      if (cmd & kCmdKFinal) tc_commit(&ctrl.ring_empty[k_slot]);
       if (cmd & kCmdQEnd) tc_commit(&ctrl.q_empty[s]);
     }
     if (next != 0) {
