@@ -269,8 +269,31 @@ steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy
     w.lo[1] = b ? 0 : 1;
     w.hi[1] = b ? int32_t(nb) - 1 : 0;
     w.n_steps = int32_t(std::max(na, nb));
+    // Key tiles may be visited in any order (the online softmax does not care), so the tiles both
+    // query tiles want come first, in the same steps: each of those steps needs one K/V load, not two.
+    std::vector<uint32_t> ea, eb;
+    if (b) {
+      std::vector<uint32_t> rest_a, rest_b;
+      size_t ia = 0, ib = 0;
+      while (ia < na || ib < nb) {
+        const uint32_t ta = ia < na ? (a->entries[ia] & kEntryTileMask) : 0xFFFFFFFFu;
+        const uint32_t tb = ib < nb ? (b->entries[ib] & kEntryTileMask) : 0xFFFFFFFFu;
+        if (ta == tb) {
+          ea.push_back(a->entries[ia++]);
+          eb.push_back(b->entries[ib++]);
+        } else if (ta < tb) {
+          rest_a.push_back(a->entries[ia++]);
+        } else {
+          rest_b.push_back(b->entries[ib++]);
+        }
+      }
+      ea.insert(ea.end(), rest_a.begin(), rest_a.end());
+      eb.insert(eb.end(), rest_b.begin(), rest_b.end());
+    } else {
+      ea = a->entries;
+    }
     for (size_t t = 0; t < size_t(w.n_steps); ++t)
-      d.list.push_back(StepPair{{t < na ? a->entries[t] : 0u, t < nb ? b->entries[t] : 0u}});
+      d.list.push_back(StepPair{{t < na ? ea[t] : 0u, t < nb ? eb[t] : 0u}});
     w.cost = int32_t(na + nb);
     drafts.push_back(std::move(d));
   };
@@ -304,7 +327,32 @@ steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy
       if (c.bitmap) {
         // similar lengths pair best: both tiles of an item then finish together
         std::stable_sort(live.begin(), live.end(), [](const Task *a, const Task *b) { return a->count() > b->count(); });
-        for (size_t n = 0; n < live.size(); n += 2) finish_list(live[n], n + 1 < live.size() ? live[n + 1] : nullptr, batch, g);
+        // among the next few tasks of similar length, take the partner with the most key tiles in common
+        std::vector<bool> used(live.size(), false);
+        for (size_t n = 0; n < live.size(); ++n) {
+          if (used[n]) continue;
+          used[n] = true;
+          size_t best = live.size(), seen = 0;
+          int64_t best_common = 0;
+          for (size_t m = n + 1; m < live.size() && seen < kPartnerWindow; ++m) {
+            if (used[m]) continue;
+            ++seen;
+            int64_t common = 0;
+            size_t ia = 0, ib = 0;
+            const std::vector<uint32_t> &ea = live[n]->entries, &eb = live[m]->entries;
+            while (ia < ea.size() && ib < eb.size()) {
+              const uint32_t ta = ea[ia] & kEntryTileMask, tb = eb[ib] & kEntryTileMask;
+              if (ta == tb) { ++common; ++ia; ++ib; }
+              else if (ta < tb) ++ia;
+              else ++ib;
+            }
+            // a step with one idle slot costs far more than a shared load saves
+            const int64_t score = common - 16 * (live[n]->count() - live[m]->count());
+            if (score > best_common || best == live.size()) { best_common = score; best = m; }
+          }
+          if (best < live.size()) used[best] = true;
+          finish_list(live[n], best < live.size() ? live[best] : nullptr, batch, g);
+        }
       } else if (G % 2 == 0) {
         // two query heads of the group on the same query tile: identical key ranges
         for (int h = g * G; h < (g + 1) * G; h += 2)

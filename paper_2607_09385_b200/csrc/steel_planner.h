@@ -13,6 +13,8 @@ namespace steel {
 constexpr int64_t kL2WaveBytes = 64ll << 20;
 // Fixed cost of an item (Q load, first-tile latency, epilogue) in units of one key-tile step.
 constexpr int kItemOverheadSteps = 2;
+// Bitmap masks: how many tasks of similar length are examined when choosing a query tile's partner.
+constexpr size_t kPartnerWindow = 16;
 // CTA count assumed by the host-only planning entry point (the SM count of a B200).
 constexpr int kPlanHostCtas = 148;
 
