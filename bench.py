@@ -199,6 +199,64 @@ def run_paper_sweep(args, dev):
           flush=True)
 
 
+def run_unfused_sweep(args, dev):
+    """Fused kernel against layer-by-layer attention (library GEMM -> scale/mask -> softmax -> library
+    GEMM, every intermediate through HBM) on the paper's shapes, with the modelled HBM traffic of
+    both.  The layer-by-layer arm is a comparison baseline, not part of the library."""
+    import torch
+    from paper_2607_09385_b200 import binding, traffic_model
+
+    def unfused(q, k, v, scale, causal):
+        a = torch.matmul(q, k.transpose(-1, -2))
+        a = a * scale
+        if causal:
+            s = q.shape[-2]
+            a = a.masked_fill(torch.ones(s, s, dtype=torch.bool, device=q.device).triu(1), float("-inf"))
+        p = torch.softmax(a, dim=-1, dtype=torch.float32).to(torch.bfloat16)
+        return torch.matmul(p, v)
+
+    rows = []
+    for w in inputs.paper_workloads():
+        if w.heads_q * w.seq * w.seq * 2 > (8 << 30):      # the score matrix must fit comfortably
+            continue
+        data = inputs.make_inputs(w, inputs.DEFAULT_SEED)
+        attn = binding.SteelAttention(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim, w.scale, w.flags,
+                                      w.block, w.window, None)
+        q, k, v = (torch.from_numpy(data[x].view(np.int16)).to(dev).view(torch.bfloat16) for x in "qkv")
+        o = torch.empty_like(q)
+        causal = bool(w.flags & inputs.MASK_CAUSAL)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        ms_fused = timed(lambda: attn.run(q, k, v, o, None, want_lse=False))
+        ms_unfused = timed(lambda: unfused(q, k, v, w.scale, causal))
+        ref = unfused(q, k, v, w.scale, causal)
+        err = float((ref.float() - o.float()).abs().max())
+        st = attn.stats()
+        fused_model = traffic_model.fused_bytes(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim,
+                                                st["kv_tile_loads"])
+        unfused_model = traffic_model.unfused_bytes(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim)
+        rows.append({"workload": w.name, "seq": w.seq, "ms_fused": ms_fused, "ms_layer_by_layer": ms_unfused,
+                     "speedup": ms_unfused / ms_fused, "max_abs_diff": err,
+                     "model_bytes_fused_compulsory": fused_model["compulsory"],
+                     "model_bytes_fused_no_reuse": fused_model["no_reuse"],
+                     "model_bytes_layer_by_layer": unfused_model["total"]})
+        attn.close()
+        del q, k, v, o, ref
+        torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "unfused", "steps": args.steps, "results": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -211,8 +269,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--policy", type=int, default=0)
-    ap.add_argument("--sweep", default="", choices=["", "paper"],
-                    help="'paper': time the paper's own attention shapes (head_dim 64) instead of one workload")
+    ap.add_argument("--sweep", default="", choices=["", "paper", "unfused"],
+                    help="'paper': time the paper's own attention shapes (head_dim 64) instead of one workload; "
+                         "'unfused': the same shapes against layer-by-layer attention through HBM")
     ap.add_argument("--profile-heads", type=int, default=0,
                     help="shrink the workload to this many query heads (same KV grouping) for ncu captures")
     args = ap.parse_args()
@@ -246,6 +305,9 @@ def main():
 
     if args.sweep == "paper":
         run_paper_sweep(args, dev)
+        return
+    if args.sweep == "unfused":
+        run_unfused_sweep(args, dev)
         return
 
     # every rank works on its own replica (independent problem, own seed)
