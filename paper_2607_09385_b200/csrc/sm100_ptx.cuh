@@ -110,6 +110,16 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar) {
                : "memory");
 }
 
+// The same, executed only if `enable` is non-zero (a predicated instruction, not a branch).
+__device__ __forceinline__ void tc_commit_if(uint64_t *bar, uint32_t enable) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %1, 0;\n\t"
+      "@p tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(smem_u32(bar)), "r"(enable)
+      : "memory");
+}
+
 // D[tmem] (+)= A[smem desc] * B[smem desc], bf16 operands, fp32 accumulator.
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {

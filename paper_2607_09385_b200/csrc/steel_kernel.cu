@@ -374,30 +374,30 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
     bool ok_v = !need_v || mbar_test_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u);
     bool ok_k = !need_k || mbar_test_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u);
     bool ok_p = !has_pv || mbar_test_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u);
+    // rare waits (first / last step of an item) and barriers that were not yet complete
+    constexpr uint32_t kRare = kCmdWaitOEmpty | kCmdWaitQFull | kCmdOEnd | kCmdQEnd;
+    const uint32_t rare = cmd & kRare;
+    if (rare | uint32_t(!ok_v) | uint32_t(!ok_k) | uint32_t(!ok_p)) {
+      bool ok = true;
+      if (cmd & kCmdWaitOEmpty) ok = bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status);
+      if (ok && (cmd & kCmdWaitQFull))
+        ok = bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status);
+      if (ok && !ok_v) ok = bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status);
+      if (ok && !ok_k) ok = bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status);
+      if (ok && !ok_p) ok = bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status);
+      if (!ok) break;
+    }
+    tc_fence_after();
     if (has_pv) {
-      if ((cmd & kCmdWaitOEmpty) &&
-          !bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status))
-        break;
-      if (!ok_v && !bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status)) break;
-      if (!ok_p && !bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status)) break;
-      tc_fence_after();
       const uint64_t dv = desc_v0 + uint64_t((v_slot * C::kTileBytes) >> 4);
       const uint32_t t_o = tmem + C::kColO + s * D;
       const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u;
 #pragma unroll
       for (int kk = 0; kk < kTile / 16; ++kk)
         mma_ts(t_o, t_s + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
-      if (cmd & kCmdVFinal) tc_commit(&ctrl.ring_empty[v_slot]);
-      if (cmd & kCmdOEnd) tc_commit(&ctrl.o_full[s]);
+      tc_commit_if(&ctrl.ring_empty[v_slot], cmd & kCmdVFinal);
     }
     if (has_s) {
-      if ((cmd & kCmdWaitQFull) &&
-          !bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status))
-        break;
-      if (!ok_k && !bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status)) break;
-      // after a PV of the same command the fence above still orders this product behind the
-      // softmax warps' reads of S
-      if (!has_pv) tc_fence_after();
       const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
       const uint64_t dk = desc_k0 + uint64_t((k_slot * C::kTileBytes) >> 4);
 #pragma unroll
@@ -406,8 +406,12 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
         mma_ss(t_s, dq + off, dk + off, idesc_s, kk > 0);
       }
       tc_commit(&ctrl.s_full[s]);
-      if (cmd & kCmdKFinal) tc_commit(&ctrl.ring_empty[k_slot]);
-      if (cmd & kCmdQEnd) tc_commit(&ctrl.q_empty[s]);
+      tc_commit_if(&ctrl.ring_empty[k_slot], cmd & kCmdKFinal);
+    }
+    if (rare) {
+      // all of this command's MMAs are issued: these commits cover them
+      tc_commit_if(&ctrl.o_full[s], cmd & kCmdOEnd);
+      tc_commit_if(&ctrl.q_empty[s], cmd & kCmdQEnd);
     }
     if (next != 0) {
       *next_cell = 0;
