@@ -108,7 +108,8 @@ steel_status_t steel_attn_create(const steel_attn_params_t *params, steel_attn_t
  * stream).  q, k, v, o: device bf16 tensors in the layouts above; lse: device float32 or
  * NULL.  Asynchronous: no allocation, no host synchronisation.  One persistent kernel is
  * launched; device-side waits are bounded and, if one expires, the kernel stops and the
- * error is reported by steel_attn_last_status.
+ * error is reported by steel_attn_last_status.  STEEL_ERR_INVALID_ARG also if the current device
+ * is not the one the handle was created on.
  */
 steel_status_t steel_attn_run(steel_attn_t *handle, const void *q, const void *k, const void *v,
                               void *o, float *lse, void *cuda_stream);

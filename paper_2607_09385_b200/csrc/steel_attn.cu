@@ -168,6 +168,9 @@ steel_status_t steel_attn_run(steel_attn_t *h, const void *q, const void *k, con
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3u))
     return STEEL_ERR_INVALID_ARG;
   const steel_attn_params_t &p = h->params;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return STEEL_ERR_CUDA;
+  if (device != h->device) return STEEL_ERR_INVALID_ARG;  // the work lists live on the create-time device
   CUtensorMap map_q, map_k, map_v;
   if (!make_map(&map_q, q, p.head_dim, p.seq_q, int64_t(p.batch) * p.heads_q) ||
       !make_map(&map_k, k, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv) ||
