@@ -5,16 +5,19 @@
 //   warps 0-3 / 4-7 : softmax warpgroup of slot 0 / 1.  Thread r owns query row r: it reads the
 //                     score row S (fp32) from TMEM, applies scale and (partial tiles only) the mask
 //                     computed from coordinates, keeps the running maximum m and sum l, writes
-//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S, rescales O when the maximum has grown,
-//                     and at the end writes O / l and LSE.  (Algorithm 1: scale_and_mask and rowmax of
-//                     the First Stage, the Second Stage, and the rescale of the Third.)
-//   warp 8          : TMA producer.  Loads Q once per item and K_j / V_j for executed tiles only into
-//                     a shared-memory ring; a tile wanted by both slots in the same step is loaded once.
-//   warp 9          : MMA issuer.  S = Q K^T (both operands in shared memory) and O += P V (P from
-//                     TMEM, V from shared memory) on tcgen05 with fp32 accumulators in TMEM.
-// Producer and MMA issuer enumerate an item's operations with the same generator (Walker), so ring
-// positions agree without communication.  Every mbarrier wait is bounded; on expiry the CTA sets
-// the status word and all roles leave.
+//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S, rescales O when the
+//                     maximum has grown, and at the end writes O / l and LSE.  (Algorithm 1:
+//                     scale_and_mask and rowmax of the First Stage, the Second Stage, and the rescale
+//                     of the Third.)
+//   warp 8          : TMA producer and scheduler.  Walks the items, loads Q once per item and K_j / V_j
+//                     for executed tiles only into a shared-memory ring (a tile wanted by both slots
+//                     in the same step is loaded once), and publishes one command word per slot-step
+//                     for the MMA issuer, with ring slots, barrier phases and release flags worked out.
+//   warp 9          : MMA issuer.  Pops commands and issues S = Q K^T (both operands in shared memory)
+//                     and O += P V (P from TMEM, V from shared memory) on tcgen05 with fp32
+//                     accumulators in TMEM.  Its loop time is the kernel's period, so it does nothing else.
+//   warps 10-11     : idle (they only keep the warpgroup complete for the register re-split).
+// Every mbarrier and queue wait is bounded; on expiry the CTA sets the status word and all roles leave.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
