@@ -149,7 +149,8 @@ __device__ __forceinline__ uint2 load_step(const Item &w, const StepPair *steps,
 }
 
 // The canonical order of an item's tensor-core operations S(s, t) = Q_s K_j^T and PV(s, t):
-// O_s += P_s V_j, shared by the producer (which loads a tile at its first use) and the MMA issuer.
+// O_s += P_s V_j: the order in which the producer loads tiles (at their first use) and publishes
+// commands, and therefore the order in which the MMA issuer executes them.
 // For each step t: first S(s, t) of slots that start at t, then for each present slot PV(s, t)
 // followed by S(s, t + 1).  A tile wanted by both slots in one step is one ring fill: slot 0 uses
 // it first, slot 1 last (the planner guarantees lo0 <= lo1).  `ring` counts fills.
@@ -253,7 +254,8 @@ __device__ __forceinline__ uint32_t fifo_pop(Ctrl &ctrl, uint32_t &head, int32_t
 }
 
 // The producer is also the scheduler: it walks the items, issues the TMA loads and publishes one
-// command word per tensor-core operation, so the MMA issuer's own loop stays a few instructions long.
+// command word per slot-step (PV(s, t) fused with the S(s, t + 1) that follows it), so the MMA
+// issuer's own loop stays a few instructions long.
 template <int D>
 __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, const CUtensorMap *map_k,
                               const CUtensorMap *map_v, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring) {
