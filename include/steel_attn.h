@@ -180,6 +180,44 @@ steel_status_t steel_attn_set_policy(int32_t policy);
 steel_status_t steel_attn_run_noalloc(const steel_attn_params_t *params, const void *q, const void *k,
                                       const void *v, void *o, float *lse, void *cuda_stream);
 
+/*
+ * The same operation for tensors in HOST memory (the end-to-end path of Eq. 1 / Algorithm 1:
+ * operands start and results end on the host).  A host-side object owns device staging buffers for
+ * Q, K, V, O and LSE, three internal streams and one plan per chunk.  The problem is cut into at
+ * most `max_chunks` chunks that are independent attention problems with contiguous tensors: groups
+ * of batch elements when batch > 1, groups of KV heads (with their query heads and their slice of
+ * the bitmap) when batch == 1; the number used is the largest divisor of batch (of heads_kv) not
+ * above max_chunks (values below 1 mean 1).  Chunk c is copied host -> device, run through the
+ * kernel of steel_attn_run and copied device -> host on separate streams, so the copies of one
+ * chunk overlap the kernel of another.  Results equal those of steel_attn_run on the same chunk.
+ */
+typedef struct steel_attn_host steel_attn_host_t; /* opaque, owned by the library */
+
+/* Plan the chunks, allocate the staging buffers (the size of all five tensors) on the current
+ * device.  Status codes as for steel_attn_create; *out is NULL on failure. */
+steel_status_t steel_attn_host_create(const steel_attn_params_t *params, int32_t max_chunks,
+                                      steel_attn_host_t **out);
+
+/*
+ * q, k, v (read) and o, lse (written; lse may be NULL) are HOST pointers in the layouts above, owned
+ * by the caller and valid until `cuda_stream` has executed the call.  With page-locked host memory
+ * the call is asynchronous; with pageable memory the copies block the calling thread but the result
+ * is the same.  The work is ordered after what is already queued on `cuda_stream`, and later work on
+ * `cuda_stream` is ordered after the last device -> host copy.  One object must not be used from
+ * two streams or threads at once (the staging buffers are shared between its calls).
+ */
+steel_status_t steel_attn_host_run(steel_attn_host_t *handle, const void *q, const void *k,
+                                   const void *v, void *o, float *lse, void *cuda_stream);
+
+/* Synchronise `cuda_stream`, then report and clear the device status of the chunks' kernels. */
+steel_status_t steel_attn_host_last_status(steel_attn_host_t *handle, void *cuda_stream);
+
+/* Number of chunks the object uses (0 for NULL). */
+int32_t steel_attn_host_chunks(const steel_attn_host_t *handle);
+
+/* Wait for the object's streams, release its plans, buffers, streams and events. NULL is STEEL_OK. */
+steel_status_t steel_attn_host_destroy(steel_attn_host_t *handle);
+
 const char *steel_status_string(steel_status_t status);
 
 #ifdef __cplusplus

@@ -1,7 +1,8 @@
 """ctypes binding of the C ABI in ``include/steel_attn.h`` (argument marshalling only).
 
 Every function here has the name and meaning of its C counterpart; tensors are passed as raw
-device pointers taken from torch tensors, the stream as ``torch.cuda.current_stream()``.
+device pointers taken from torch tensors (host pointers for the ``steel_attn_host_*`` calls), the
+stream as ``torch.cuda.current_stream()``.
 There is no fallback: if the shared library is missing and cannot be built, importing the
 binding's functions raises.
 """
@@ -22,6 +23,8 @@ EXPORTS = (
     "steel_attn_create", "steel_attn_run", "steel_attn_last_status", "steel_attn_destroy",
     "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_set_policy", "steel_attn_run_noalloc",
     "steel_attn_debug_stall",
+    "steel_attn_host_create", "steel_attn_host_run", "steel_attn_host_last_status", "steel_attn_host_chunks",
+    "steel_attn_host_destroy",
     "steel_status_string",
 )
 
@@ -86,6 +89,11 @@ def load_library():
     lib.steel_attn_set_policy.argtypes = [ctypes.c_int32]
     lib.steel_attn_debug_stall.argtypes = [vp, ctypes.c_int32, ctypes.c_int64]
     lib.steel_attn_run_noalloc.argtypes = [ctypes.POINTER(Params), vp, vp, vp, vp, vp, vp]
+    lib.steel_attn_host_create.argtypes = [ctypes.POINTER(Params), ctypes.c_int32, ctypes.POINTER(vp)]
+    lib.steel_attn_host_run.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.steel_attn_host_last_status.argtypes = [vp, vp]
+    lib.steel_attn_host_chunks.argtypes = [vp]
+    lib.steel_attn_host_destroy.argtypes = [vp]
     lib.steel_status_string.argtypes = [ctypes.c_int]
     lib.steel_status_string.restype = ctypes.c_char_p
     for name in EXPORTS[:-1]:
@@ -176,6 +184,35 @@ def steel_attn_set_policy(policy: int) -> None:
         raise SteelError(st, "steel_attn_set_policy")
 
 
+def steel_attn_host_create(params: Params, max_chunks: int) -> int:
+    handle = ctypes.c_void_p()
+    st = load_library().steel_attn_host_create(ctypes.byref(params), max_chunks, ctypes.byref(handle))
+    if st != STEEL_OK:
+        raise SteelError(st, "steel_attn_host_create")
+    return handle.value
+
+
+def steel_attn_host_run(handle: int, q_ptr: int, k_ptr: int, v_ptr: int, o_ptr: int, lse_ptr, stream: int) -> None:
+    """All five pointers are HOST addresses (page-locked memory makes the call asynchronous)."""
+    st = load_library().steel_attn_host_run(handle, q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, stream)
+    if st != STEEL_OK:
+        raise SteelError(st, "steel_attn_host_run")
+
+
+def steel_attn_host_last_status(handle: int, stream: int) -> int:
+    return load_library().steel_attn_host_last_status(handle, stream)
+
+
+def steel_attn_host_chunks(handle: int) -> int:
+    return load_library().steel_attn_host_chunks(handle)
+
+
+def steel_attn_host_destroy(handle) -> None:
+    st = load_library().steel_attn_host_destroy(handle)
+    if st != STEEL_OK:
+        raise SteelError(st, "steel_attn_host_destroy")
+
+
 class SteelAttention:
     """Convenience owner of one handle: ``SteelAttention(...).run(q, k, v)`` on CUDA torch tensors."""
 
@@ -211,6 +248,50 @@ class SteelAttention:
     def close(self) -> None:
         if self.handle:
             steel_attn_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class SteelAttentionHost:
+    """Owner of one host-memory attention object: ``run`` takes CPU torch tensors (bf16 bit patterns
+    as int16 or bfloat16; page-locked for overlap) and fills ``o`` / ``lse`` in host memory."""
+
+    def __init__(self, batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, flags=0, block=128,
+                 window=0, bitmap=None, max_chunks=4):
+        self.params, self._keep = make_params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale,
+                                              flags, block, block, window, bitmap)
+        self.shape_q = (batch, heads_q, seq_q, head_dim)
+        self.shape_kv = (batch, heads_kv, seq_kv, head_dim)
+        self.handle = steel_attn_host_create(self.params, max_chunks)
+
+    @property
+    def chunks(self) -> int:
+        return steel_attn_host_chunks(self.handle)
+
+    def run(self, q, k, v, o, lse=None):
+        import torch
+        for t, shape in ((q, self.shape_q), (k, self.shape_kv), (v, self.shape_kv), (o, self.shape_q)):
+            assert not t.is_cuda and t.element_size() == 2 and t.is_contiguous() and tuple(t.shape) == shape
+        if lse is not None:
+            assert (not lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+                    and tuple(lse.shape) == self.shape_q[:3])
+        stream = torch.cuda.current_stream().cuda_stream
+        steel_attn_host_run(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                            lse.data_ptr() if lse is not None else None, stream)
+        return o, lse
+
+    def last_status(self) -> int:
+        import torch
+        return steel_attn_host_last_status(self.handle, torch.cuda.current_stream().cuda_stream)
+
+    def close(self) -> None:
+        if self.handle:
+            steel_attn_host_destroy(self.handle)
             self.handle = None
 
     def __del__(self):

@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libsteel_attn.so")
-SOURCES = ("steel_attn.cu", "steel_kernel.cu", "steel_noalloc.cu", "steel_planner.cpp")
+SOURCES = ("steel_attn.cu", "steel_kernel.cu", "steel_noalloc.cu", "steel_host.cu", "steel_planner.cpp")
 HEADERS = ("sm100_ptx.cuh", "steel_kernel.h", "steel_plan.h", "steel_planner.h")
 NVCC_FLAGS = ("-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-cudart", "static")
