@@ -72,3 +72,23 @@ def test_create_without_gpu_fails_loudly():
     handle = ctypes.c_void_p(123)
     st = B.load_library().steel_attn_create(ctypes.byref(p), ctypes.byref(handle))
     assert st == B.STEEL_ERR_CUDA and handle.value is None
+
+
+def test_host_entry_points_argument_checks_and_no_gpu():
+    """The host-memory form validates before touching CUDA and has no CPU fallback either."""
+    lib = B.load_library()
+    handle = ctypes.c_void_p(123)
+    assert lib.steel_attn_host_create(None, 4, ctypes.byref(handle)) == B.STEEL_ERR_INVALID_ARG
+    assert handle.value is None
+    p, _ = B.make_params(1, 4, 3, 256, 256, 64, 0.125, 1, 64, 64)  # heads_q % heads_kv != 0
+    assert lib.steel_attn_host_create(ctypes.byref(p), 4, ctypes.byref(handle)) == B.STEEL_ERR_INVALID_ARG
+    assert lib.steel_attn_host_create(ctypes.byref(p), 4, None) == B.STEEL_ERR_INVALID_ARG
+    assert lib.steel_attn_host_run(None, None, None, None, None, None, None) == B.STEEL_ERR_INVALID_ARG
+    assert lib.steel_attn_host_last_status(None, None) == B.STEEL_ERR_INVALID_ARG
+    assert lib.steel_attn_host_chunks(None) == 0
+    assert lib.steel_attn_host_destroy(None) == B.STEEL_OK
+    if not torch.cuda.is_available():
+        p, _ = B.make_params(2, 2, 2, 256, 256, 64, 0.125, 1, 64, 64)
+        handle = ctypes.c_void_p(123)
+        st = lib.steel_attn_host_create(ctypes.byref(p), 2, ctypes.byref(handle))
+        assert st == B.STEEL_ERR_CUDA and handle.value is None
