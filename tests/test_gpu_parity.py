@@ -126,6 +126,38 @@ def test_seq_q_differs_from_seq_kv():
         attn.close()
 
 
+RECT_CASES = [
+    # name, seq_q, seq_kv, head_dim, heads_q, heads_kv, flags, window, scale
+    ("decode_like_one_query", 1, 3000, 128, 4, 2, CAUSAL, 0, 0.09),
+    ("decode_like_window", 5, 2000, 64, 2, 2, CAUSAL | WINDOW, 700, 0.125),
+    ("cross_attention_dense", 300, 1000, 128, 2, 1, 0, 0, 0.09),
+    ("window_longer_than_sequence", 640, 640, 128, 2, 2, CAUSAL | WINDOW, 100000, 0.09),
+    ("large_scale", 384, 384, 64, 2, 2, CAUSAL, 0, 1.5),
+]
+
+
+@pytest.mark.parametrize("case", RECT_CASES, ids=[c[0] for c in RECT_CASES])
+def test_rectangular_and_degenerate_shapes(case):
+    """Few queries against many keys (bottom-right aligned masks), unmasked cross attention, a window
+    that never cuts, and a softmax scale that makes the exponents large: every row against the oracle."""
+    import oracle
+    name, sq, skv, D, Hq, Hkv, flags, window, scale = case
+    rng = np.random.default_rng(len(name))
+    q = inputs.f32_to_bf16_bits(rng.standard_normal((1, Hq, sq, D)).astype(np.float32))
+    k = inputs.f32_to_bf16_bits(rng.standard_normal((1, Hkv, skv, D)).astype(np.float32))
+    v = inputs.f32_to_bf16_bits(rng.standard_normal((1, Hkv, skv, D)).astype(np.float32))
+    attn = binding.SteelAttention(1, Hq, Hkv, sq, skv, D, scale, flags, window=window)
+    o, lse = attn.run(H.to_device(q), H.to_device(k), H.to_device(v))
+    assert attn.last_status() == binding.STEEL_OK
+    p = oracle.OracleProblem(1, Hq, Hkv, sq, skv, D, scale, flags, 128, 128, window)
+    o_ref, lse_ref = oracle.rows(p, q, k, v, oracle.steel_oracle.all_rows(p))
+    og, lg = o.float().cpu().numpy().reshape(-1, D), lse.cpu().numpy().reshape(-1)
+    assert np.isfinite(lse_ref).all() and np.isfinite(lg).all()
+    err = np.abs(og - o_ref)
+    assert err.max() <= H.TOL_O_MAX and err.mean() <= H.TOL_O_MEAN and np.abs(lg - lse_ref).max() <= H.TOL_LSE
+    attn.close()
+
+
 def test_bitmap_with_empty_row_blocks():
     """Rows whose bitmap row-block is empty: O = 0 and LSE = -inf, neighbours unaffected."""
     w = inputs.Workload("empty_rows", 1, 2, 2, 512, 128, 128, BITMAP)
