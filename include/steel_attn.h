@@ -31,7 +31,7 @@
  * Ownership and threading: every tensor pointer is a DEVICE pointer owned by the caller,
  * 16-byte aligned, and must stay valid until the stream has executed the call.  The bitmap
  * is a HOST pointer read only during steel_attn_create.  A handle owns its device work lists
- * and scheduler counter; it is bound to the device that was current at create time and must
+ * and status word; it is bound to the device that was current at create time and must
  * not be used by two streams at once.  All functions return a status code; nothing throws,
  * aborts or traps.  There is no CPU fallback: without a usable CUDA device the run fails.
  */
@@ -72,6 +72,19 @@ typedef struct {
   int32_t head_dim;                 /* 64 or 128                                                 */
   float scale;                      /* finite, > 0; multiplies q.k before softmax                */
   steel_mask_desc_t mask;
+  int32_t policy;                   /* placement of query tiles on the persistent CTAs (paper Sec.
+                                       "Sparsity-Aware Pipeline Placement"): 0 = query tiles paired for
+                                       shared K/V loads, items ordered KV-head-major then longest first,
+                                       each to the least loaded CTA (default); 1 = the same items in
+                                       natural order cut into contiguous chunks, one per CTA (the paper's
+                                       "uniform placement"); 2 = the same items dealt round-robin to the
+                                       CTAs (the paper's sparsity-aware placement: consecutive query
+                                       tiles side by side)                                         */
+  int32_t exp_emulation;            /* share of the Second Stage's exponentials evaluated by a cubic
+                                       polynomial on the FMA pipe instead of the special-function unit
+                                       (the counterpart of the lookup-table exponent of the paper's Sec.
+                                       "Comparison with State-of-the-Art on NPU"): 0 = none (default),
+                                       1 = 12.5 %, 2 = 25 %, 3 = 50 %; relative error 7.5e-5 per value  */
 } steel_attn_params_t;
 
 /* Work-list statistics of a plan (the skip set of the three mask cases, at the kernel's
@@ -104,7 +117,7 @@ typedef struct {
 steel_status_t steel_attn_create(const steel_attn_params_t *params, steel_attn_t **out);
 
 /*
- * Enqueue one attention call on `cuda_stream` (a cudaStream_t cast to void*; NULL = default
+ * Enqueue one attention call (Eq. 1, computed as Algorithm 1 over the handle's work lists) on `cuda_stream` (a cudaStream_t cast to void*; NULL = default
  * stream).  q, k, v, o: device bf16 tensors in the layouts above; lse: device float32 or
  * NULL.  Asynchronous: no allocation, no host synchronisation.  One persistent kernel is
  * launched; device-side waits are bounded and, if one expires, the kernel stops and the
@@ -116,11 +129,12 @@ steel_status_t steel_attn_run(steel_attn_t *handle, const void *q, const void *k
 
 /*
  * Synchronise `cuda_stream` and report the device-side status word of the handle's last
- * runs (STEEL_OK or STEEL_ERR_TIMEOUT), then clear it.
+ * runs of Algorithm 1's pipeline (its stages hand tiles over through bounded waits) (STEEL_OK or STEEL_ERR_TIMEOUT), then clear it.
  */
 steel_status_t steel_attn_last_status(steel_attn_t *handle, void *cuda_stream);
 
-/* Release the handle and its device memory.  destroy(NULL) is STEEL_OK. */
+/* Release the handle and the device work lists built from the mask cases of Sec. "The STEEL
+ * Pipeline".  destroy(NULL) is STEEL_OK. */
 steel_status_t steel_attn_destroy(steel_attn_t *handle);
 
 /* Statistics of the handle's plan. */
@@ -146,14 +160,14 @@ steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_att
  */
 steel_status_t steel_attn_debug_stall(steel_attn_t *handle, int32_t cta, int64_t timeout_cycles);
 
-/* Number of scheduler policies and selection of one for subsequently created handles
- * (process-wide; default 0).  0: query tiles paired for shared K/V loads, items ordered
- * KV-head-major then longest first (the sparsity-aware placement idea of the paper's Sec.
- * "Sparsity-Aware Pipeline Placement" recast for persistent CTAs); 1: the same items in natural
- * order cut into contiguous chunks, one per CTA (the paper's "uniform placement"); 2: the same
- * items dealt round-robin to the CTAs (the paper's sparsity-aware placement: consecutive query
- * tiles side by side). */
-steel_status_t steel_attn_set_policy(int32_t policy);
+/*
+ * Measurement hook for the roofline figures (paper Sec. "Attention Benchmark": throughput is quoted
+ * against the device's peak, which depends on the clock actually held).  With a non-NULL
+ * `device_pair` (DEVICE pointer to two int64, 8-byte aligned, owned by the caller), CTA 0 of each of
+ * the handle's following runs stores {SM cycles, nanoseconds} elapsed over its run there, so that
+ * cycles / nanoseconds is the SM clock in GHz during the kernel.  NULL switches the hook off.
+ */
+steel_status_t steel_attn_debug_clock_probe(steel_attn_t *handle, int64_t *device_pair);
 
 /*
  * (The paper has no counterpart to this entry point; it exists for integration.)  One attention
@@ -167,7 +181,7 @@ steel_status_t steel_attn_set_policy(int32_t policy);
  * Limits: at most 16384 work items, 131072 explicit step-list entries (bitmap masks) and 1024
  * persistent CTAs; a problem whose plan is larger is refused with STEEL_ERR_UNSUPPORTED and
  * nothing is launched (the 131072-token graded configuration, 16384 items, is the largest
- * causal case that fits).  Arguments as for steel_attn_run; scheduling policy 0 is always used.
+ * causal case that fits).  Arguments as for steel_attn_create and steel_attn_run.
  *
  * The call is blocking: it plans on the host (transient host memory only), copies the lists on
  * `cuda_stream`, runs the kernel, waits for the stream and returns the device status (STEEL_OK or

@@ -21,8 +21,8 @@ STEEL_MASK_CAUSAL, STEEL_MASK_WINDOW, STEEL_MASK_BITMAP = 1, 2, 4
 
 EXPORTS = (
     "steel_attn_create", "steel_attn_run", "steel_attn_last_status", "steel_attn_destroy",
-    "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_set_policy", "steel_attn_run_noalloc",
-    "steel_attn_debug_stall",
+    "steel_attn_get_stats", "steel_attn_plan_host", "steel_attn_run_noalloc",
+    "steel_attn_debug_stall", "steel_attn_debug_clock_probe",
     "steel_attn_host_create", "steel_attn_host_run", "steel_attn_host_last_status", "steel_attn_host_chunks",
     "steel_attn_host_destroy",
     "steel_status_string",
@@ -37,7 +37,8 @@ class MaskDesc(ctypes.Structure):
 class Params(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("heads_q", ctypes.c_int32), ("heads_kv", ctypes.c_int32),
                 ("seq_q", ctypes.c_int32), ("seq_kv", ctypes.c_int32), ("head_dim", ctypes.c_int32),
-                ("scale", ctypes.c_float), ("mask", MaskDesc)]
+                ("scale", ctypes.c_float), ("mask", MaskDesc), ("policy", ctypes.c_int32),
+                ("exp_emulation", ctypes.c_int32)]
 
 
 class Stats(ctypes.Structure):
@@ -86,8 +87,8 @@ def load_library():
     lib.steel_attn_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
     lib.steel_attn_plan_host.argtypes = [ctypes.POINTER(Params), ctypes.POINTER(Stats), vp, ctypes.c_int64,
                                          ctypes.POINTER(ctypes.c_int64)]
-    lib.steel_attn_set_policy.argtypes = [ctypes.c_int32]
     lib.steel_attn_debug_stall.argtypes = [vp, ctypes.c_int32, ctypes.c_int64]
+    lib.steel_attn_debug_clock_probe.argtypes = [vp, vp]
     lib.steel_attn_run_noalloc.argtypes = [ctypes.POINTER(Params), vp, vp, vp, vp, vp, vp]
     lib.steel_attn_host_create.argtypes = [ctypes.POINTER(Params), ctypes.c_int32, ctypes.POINTER(vp)]
     lib.steel_attn_host_run.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -103,7 +104,7 @@ def load_library():
 
 
 def make_params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, flags=0, block_q=128,
-                block_kv=128, window=0, bitmap=None):
+                block_kv=128, window=0, bitmap=None, policy=0, exp_emulation=0):
     """Build a ``steel_attn_params_t``; returns (params, keepalive) where keepalive holds the
     host bitmap array the descriptor points to."""
     keep = None
@@ -112,7 +113,7 @@ def make_params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, flags=
         keep = np.ascontiguousarray(bitmap, dtype=np.uint32)
         ptr = keep.ctypes.data
     mask = MaskDesc(flags, block_q, block_kv, window, ptr)
-    return Params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, mask), keep
+    return Params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, mask, policy, exp_emulation), keep
 
 
 def steel_status_string(status: int) -> str:
@@ -178,10 +179,10 @@ def steel_attn_debug_stall(handle: int, cta: int, timeout_cycles: int = 0) -> No
         raise SteelError(st, "steel_attn_debug_stall")
 
 
-def steel_attn_set_policy(policy: int) -> None:
-    st = load_library().steel_attn_set_policy(policy)
+def steel_attn_debug_clock_probe(handle: int, device_pair_ptr) -> None:
+    st = load_library().steel_attn_debug_clock_probe(handle, device_pair_ptr)
     if st != STEEL_OK:
-        raise SteelError(st, "steel_attn_set_policy")
+        raise SteelError(st, "steel_attn_debug_clock_probe")
 
 
 def steel_attn_host_create(params: Params, max_chunks: int) -> int:
@@ -217,9 +218,9 @@ class SteelAttention:
     """Convenience owner of one handle: ``SteelAttention(...).run(q, k, v)`` on CUDA torch tensors."""
 
     def __init__(self, batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, flags=0, block=128,
-                 window=0, bitmap=None):
+                 window=0, bitmap=None, policy=0, exp_emulation=0):
         self.params, self._keep = make_params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale,
-                                              flags, block, block, window, bitmap)
+                                              flags, block, block, window, bitmap, policy, exp_emulation)
         self.shape_q = (batch, heads_q, seq_q, head_dim)
         self.shape_kv = (batch, heads_kv, seq_kv, head_dim)
         self.handle = steel_attn_create(self.params)
@@ -262,9 +263,9 @@ class SteelAttentionHost:
     as int16 or bfloat16; page-locked for overlap) and fills ``o`` / ``lse`` in host memory."""
 
     def __init__(self, batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale, flags=0, block=128,
-                 window=0, bitmap=None, max_chunks=4):
+                 window=0, bitmap=None, max_chunks=4, policy=0, exp_emulation=0):
         self.params, self._keep = make_params(batch, heads_q, heads_kv, seq_q, seq_kv, head_dim, scale,
-                                              flags, block, block, window, bitmap)
+                                              flags, block, block, window, bitmap, policy, exp_emulation)
         self.shape_q = (batch, heads_q, seq_q, head_dim)
         self.shape_kv = (batch, heads_kv, seq_kv, head_dim)
         self.handle = steel_attn_host_create(self.params, max_chunks)

@@ -2,7 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
-#include <atomic>
+#include <algorithm>
 #include <cstring>
 #include <limits>
 #include <new>
@@ -12,6 +12,8 @@
 #include "steel_planner.h"
 
 using namespace steel;
+
+static_assert(sizeof(steel_mask_desc_t) == 32 && sizeof(steel_attn_params_t) == 72, "public struct layout");
 
 struct steel_attn {
   steel_attn_params_t params;
@@ -23,13 +25,13 @@ struct steel_attn {
   StepPair *d_steps = nullptr;
   int32_t *d_status = nullptr;
   long long *d_trace = nullptr;  // debug builds only
+  long long *d_clock_probe = nullptr;
   long long timeout_cycles = kDefaultTimeoutCycles;
   int32_t stall_cta = -1;
+  TensorMaps maps;  // of the last (q, k, v) triple run on this handle
 };
 
 namespace {
-
-std::atomic<int> g_policy{0};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -76,15 +78,23 @@ void free_device(steel_attn *h) {
 
 namespace steel {
 
-// Encode the tensor maps for (q, k, v), fill the problem fields of `kp` (whose list and status
-// pointers the caller has set) and enqueue the kernel.
+// Encode the tensor maps for (q, k, v) unless `cache` holds them already, fill the problem fields
+// of `kp` (whose list and status pointers the caller has set) and enqueue the kernel.
 steel_status_t launch_with_params(const steel_attn_params_t &p, KernelParams kp, int grid, const void *q,
-                                  const void *k, const void *v, void *o, float *lse, cudaStream_t stream) {
-  CUtensorMap map_q, map_k, map_v;
-  if (!make_map(&map_q, q, p.head_dim, p.seq_q, int64_t(p.batch) * p.heads_q) ||
-      !make_map(&map_k, k, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv) ||
-      !make_map(&map_v, v, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv))
-    return STEEL_ERR_CUDA;
+                                  const void *k, const void *v, void *o, float *lse, cudaStream_t stream,
+                                  TensorMaps *cache) {
+  TensorMaps local;
+  TensorMaps &m = cache ? *cache : local;
+  if (m.q_ptr != q || m.k_ptr != k || m.v_ptr != v) {
+    m.q_ptr = m.k_ptr = m.v_ptr = nullptr;
+    if (!make_map(&m.q, q, p.head_dim, p.seq_q, int64_t(p.batch) * p.heads_q) ||
+        !make_map(&m.k, k, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv) ||
+        !make_map(&m.v, v, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv))
+      return STEEL_ERR_CUDA;
+    m.q_ptr = q;
+    m.k_ptr = k;
+    m.v_ptr = v;
+  }
   kp.o = o;
   kp.lse = lse;
   kp.heads_q = p.heads_q;
@@ -92,10 +102,12 @@ steel_status_t launch_with_params(const steel_attn_params_t &p, KernelParams kp,
   kp.seq_q = p.seq_q;
   kp.seq_kv = p.seq_kv;
   kp.mask_flags = p.mask.flags;
-  kp.window = int32_t(p.mask.window > std::numeric_limits<int32_t>::max() ? std::numeric_limits<int32_t>::max()
-                                                                          : p.mask.window);
+  // a window wider than the key sequence hides nothing: clamp it so that the kernel's 32-bit
+  // column arithmetic cannot overflow
+  kp.window = int32_t(std::min<int64_t>(p.mask.window, int64_t(std::max(p.seq_q, p.seq_kv)) + kTile));
   kp.scale_log2 = p.scale * 1.4426950408889634f;
-  if (launch_attention(p.head_dim, map_q, map_k, map_v, kp, grid, stream) != cudaSuccess) return STEEL_ERR_CUDA;
+  if (launch_attention(p.head_dim, p.exp_emulation, m.q, m.k, m.v, kp, grid, stream) != cudaSuccess)
+    return STEEL_ERR_CUDA;
   return STEEL_OK;
 }
 
@@ -119,7 +131,7 @@ steel_status_t steel_attn_create(const steel_attn_params_t *params, steel_attn_t
 
   Plan plan;
   try {
-    st = build_plan(params, prop.multiProcessorCount, g_policy.load(), &plan);
+    st = build_plan(params, prop.multiProcessorCount, &plan);
   } catch (const std::bad_alloc &) {
     return STEEL_ERR_ALLOC;
   }
@@ -167,37 +179,19 @@ steel_status_t steel_attn_run(steel_attn_t *h, const void *q, const void *k, con
   if (!h || !q || !k || !v || !o) return STEEL_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || (reinterpret_cast<uintptr_t>(lse) & 3u))
     return STEEL_ERR_INVALID_ARG;
-  const steel_attn_params_t &p = h->params;
   int device = -1;
   if (cudaGetDevice(&device) != cudaSuccess) return STEEL_ERR_CUDA;
   if (device != h->device) return STEEL_ERR_INVALID_ARG;  // the work lists live on the create-time device
-  CUtensorMap map_q, map_k, map_v;
-  if (!make_map(&map_q, q, p.head_dim, p.seq_q, int64_t(p.batch) * p.heads_q) ||
-      !make_map(&map_k, k, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv) ||
-      !make_map(&map_v, v, p.head_dim, p.seq_kv, int64_t(p.batch) * p.heads_kv))
-    return STEEL_ERR_CUDA;
-  KernelParams kp;
+  KernelParams kp{};
   kp.items = h->d_items;
   kp.cta_begin = h->d_cta_begin;
   kp.steps = h->d_steps;
-  kp.o = o;
-  kp.lse = lse;
   kp.status = h->d_status;
-  kp.heads_q = p.heads_q;
-  kp.heads_kv = p.heads_kv;
-  kp.seq_q = p.seq_q;
-  kp.seq_kv = p.seq_kv;
-  kp.mask_flags = p.mask.flags;
-  kp.window = int32_t(p.mask.window > std::numeric_limits<int32_t>::max() ? std::numeric_limits<int32_t>::max()
-                                                                          : p.mask.window);
-  kp.scale_log2 = p.scale * 1.4426950408889634f;
   kp.trace = h->d_trace;
+  kp.clock_probe = h->d_clock_probe;
   kp.timeout_cycles = h->timeout_cycles;
   kp.stall_cta = h->stall_cta;
-  if (launch_attention(p.head_dim, map_q, map_k, map_v, kp, h->grid, static_cast<cudaStream_t>(cuda_stream)) !=
-      cudaSuccess)
-    return STEEL_ERR_CUDA;
-  return STEEL_OK;
+  return launch_with_params(h->params, kp, h->grid, q, k, v, o, lse, static_cast<cudaStream_t>(cuda_stream), &h->maps);
 }
 
 steel_status_t steel_attn_last_status(steel_attn_t *h, void *cuda_stream) {
@@ -230,7 +224,7 @@ steel_status_t steel_attn_plan_host(const steel_attn_params_t *params, steel_att
   Plan plan;
   steel_status_t st;
   try {
-    st = build_plan(params, kPlanHostCtas, g_policy.load(), &plan);
+    st = build_plan(params, kPlanHostCtas, &plan);
   } catch (const std::bad_alloc &) {
     return STEEL_ERR_ALLOC;
   }
@@ -265,16 +259,16 @@ steel_status_t steel_attn_set_trace(steel_attn_t *h, long long *device_buffer) {
 }
 #endif
 
+steel_status_t steel_attn_debug_clock_probe(steel_attn_t *h, int64_t *device_pair) {
+  if (!h || (reinterpret_cast<uintptr_t>(device_pair) & 7u)) return STEEL_ERR_INVALID_ARG;
+  h->d_clock_probe = reinterpret_cast<long long *>(device_pair);
+  return STEEL_OK;
+}
+
 steel_status_t steel_attn_debug_stall(steel_attn_t *h, int32_t cta, int64_t timeout_cycles) {
   if (!h || cta >= h->grid) return STEEL_ERR_INVALID_ARG;
   h->stall_cta = cta < 0 ? -1 : cta;
   h->timeout_cycles = timeout_cycles > 0 ? timeout_cycles : kDefaultTimeoutCycles;
-  return STEEL_OK;
-}
-
-steel_status_t steel_attn_set_policy(int32_t policy) {
-  if (policy < 0 || policy > 2) return STEEL_ERR_INVALID_ARG;
-  g_policy.store(policy);
   return STEEL_OK;
 }
 

@@ -3,12 +3,12 @@
 // A CTA processes work items; an item is one or two query tiles (128 rows each, "slots") that walk
 // the same sequence of key-tile steps.  Roles (three warpgroups, register file re-split between them):
 //   warps 0-3 / 4-7 : softmax warpgroup of slot 0 / 1.  Thread r owns query row r: it reads the
-//                     score row S (fp32) from TMEM, applies scale and (partial tiles only) the mask
-//                     computed from coordinates, keeps the running maximum m and sum l, writes
-//                     P = 2^(S*scale*log2e - m) as bf16 back into TMEM over S, rescales O when the
-//                     maximum has grown, and at the end writes O / l and LSE.  (Algorithm 1:
-//                     scale_and_mask and rowmax of the First Stage, the Second Stage, and the rescale
-//                     of the Third.)
+//                     score row S (fp32) from TMEM into registers and hands the S buffer back,
+//                     applies scale and (partial tiles only) the mask computed from coordinates,
+//                     keeps the running maximum m and sum l, writes P = 2^(S*scale*log2e - m) as
+//                     bf16 into the slot's own P columns, rescales O when the maximum has grown, and
+//                     at the end writes O / l and LSE.  (Algorithm 1: scale_and_mask and rowmax of
+//                     the First Stage, the Second Stage, and the rescale of the Third.)
 //   warp 8          : TMA producer and scheduler.  Walks the items, loads Q once per item and K_j / V_j
 //                     for executed tiles only into a shared-memory ring (a tile wanted by both slots
 //                     in the same step is loaded once), and publishes one command word per slot-step
@@ -17,6 +17,10 @@
 //                     and O += P V (P from TMEM, V from shared memory) on tcgen05 with fp32
 //                     accumulators in TMEM.  Its loop time is the kernel's period, so it does nothing else.
 //   warps 10-11     : idle (they only keep the warpgroup complete for the register re-split).
+// Tensor memory (512 columns): one S buffer that the slots use in turn (128), P of each slot
+// (2 x 64), O of each slot (2 x head_dim).  S(s, t + 1) is issued before PV(s, t), so a slot's next
+// scores are computed while its softmax warps still work on the current tile.  (At head_dim 64 the
+// columns would allow an S buffer per slot; measured, that layout was 9 % slower.)
 // Every mbarrier and queue wait is bounded; on expiry the CTA sets the status word and all roles leave.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -35,10 +39,6 @@ constexpr int kRegsOther = 72;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;           // lazy rescale: P stays below 2^8
-#ifndef STEEL_EXP_EMULATION
-#define STEEL_EXP_EMULATION 0
-#endif
-constexpr int kExpEmulation = STEEL_EXP_EMULATION;  // 0 none, 1: 12.5 %, 2: 25 %, 3: 50 % of exp2 on the FMA pipe
 constexpr int kMaxStages = 10;
 constexpr int kFifoDepth = 32;
 constexpr uint32_t kMaskCausal = 1u, kMaskWindow = 2u;
@@ -50,13 +50,16 @@ struct Cfg {
   static constexpr int kBoxBytes = kTile * 128;
   static constexpr int kStages = (D == 128) ? 5 : 10;
   static constexpr int kSmemBytes = 1024 + (2 + kStages) * kTileBytes;
-  static constexpr uint32_t kColS = 0;    // S of slot s at columns kColS + 128 s (P aliases its first 64)
-  static constexpr uint32_t kColO = 256;  // O of slot s at columns kColO + D s
+  // Tensor-memory columns: S (fp32, 128 columns), one buffer that the slots use in turn; P of slot s
+  // (bf16 pairs, 64 columns) at kColP + 64 s; O of slot s (D columns) at kColO + D s.
+  static constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;
 };
 
 struct Ctrl {
   uint64_t ring_full[kMaxStages], ring_empty[kMaxStages];
-  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2], o_empty[2];
+  uint64_t q_full[2], q_empty[2], s_full[2], p_full[2], p_free[2], o_full[2], o_empty[2];
+  uint64_t s_free;     // the softmax warps that own the S buffer's content have it in registers
+  uint64_t drain;      // the MMA issuer's last commit when it leaves on an expired wait
   uint32_t fifo[kFifoDepth];  // command words from the producer to the MMA issuer (0 = empty)
   uint32_t tmem_base;
   int abort;
@@ -71,7 +74,7 @@ constexpr uint32_t kCmdValid = 1u << 0, kCmdHasPV = 1u << 1, kCmdHasS = 1u << 2,
                    kCmdVFinal = 1u << 16, kCmdKFinal = 1u << 17,  // last user: release the ring slot
                    kCmdWaitOEmpty = 1u << 18, kCmdOEmptyPhase = 1u << 19, kCmdWaitQFull = 1u << 20,
                    kCmdQFullPhase = 1u << 21, kCmdAcc = 1u << 22, kCmdPPhase = 1u << 23, kCmdOEnd = 1u << 24,
-                   kCmdQEnd = 1u << 25, kCmdExit = 1u << 31;
+                   kCmdQEnd = 1u << 25, kCmdWaitSFree = 1u << 26, kCmdSFreePhase = 1u << 27, kCmdExit = 1u << 31;
 
 // Optional per-role wait accounting (compiled in with -DSTEEL_TRACE only): cycles per CTA, 32 slots.
 #ifdef STEEL_TRACE
@@ -151,8 +154,10 @@ __device__ __forceinline__ uint2 load_step(const Item &w, const StepPair *steps,
 // The canonical order of an item's tensor-core operations S(s, t) = Q_s K_j^T and PV(s, t):
 // O_s += P_s V_j: the order in which the producer loads tiles (at their first use) and publishes
 // commands, and therefore the order in which the MMA issuer executes them.
-// For each step t: first S(s, t) of slots that start at t, then for each present slot PV(s, t)
-// followed by S(s, t + 1).  A tile wanted by both slots in one step is one ring fill: slot 0 uses
+// For each step t: first S(s, t) of slots that start at t, then for each present slot S(s, t + 1)
+// followed by PV(s, t): the first product runs one step ahead of the second, so a slot's next scores
+// are computed while its softmax warps still work on the current ones (they hold them in registers;
+// the S buffer in TMEM is free again as soon as they are loaded).  A tile wanted by both slots in one step is one ring fill: slot 0 uses
 // it first, slot 1 last (the planner guarantees lo0 <= lo1).  `ring` counts fills.
 // op(s, t, j, is_s, fill, first, last) returns false to stop.
 struct RingPos {
@@ -197,12 +202,12 @@ __device__ __forceinline__ bool walk_item(const Item &w, const StepPair *steps, 
     if (cur.x != 0 && t == w.lo0 && !visit(cur, 0, t, true)) return false;
     if (cur.y != 0 && t == w.lo1 && !visit(cur, 1, t, true)) return false;
     if (cur.x != 0) {
-      if (!visit(cur, 0, t, false)) return false;
       if (t < w.hi0 && !visit(nxt, 0, t + 1, true)) return false;
+      if (!visit(cur, 0, t, false)) return false;
     }
     if (cur.y != 0) {
-      if (!visit(cur, 1, t, false)) return false;
       if (t < w.hi1 && !visit(nxt, 1, t + 1, true)) return false;
+      if (!visit(cur, 1, t, false)) return false;
     }
     cur = nxt;
   }
@@ -210,7 +215,8 @@ __device__ __forceinline__ bool walk_item(const Item &w, const StepPair *steps, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Bounded push / pop of the single-producer single-consumer command queue in shared memory.
+// Bounded push into the single-producer single-consumer command queue in shared memory (the pop is
+// with the MMA issuer below).
 __device__ __forceinline__ bool fifo_push(Ctrl &ctrl, uint32_t &tail, uint32_t word, int32_t *status) {
   volatile uint32_t *cell = &ctrl.fifo[tail];
   if (*cell != 0) {
@@ -231,28 +237,6 @@ __device__ __forceinline__ bool fifo_push(Ctrl &ctrl, uint32_t &tail, uint32_t w
   tail = (tail + 1) & (kFifoDepth - 1);
   return true;
 }
-__device__ __forceinline__ uint32_t fifo_pop(Ctrl &ctrl, uint32_t &head, int32_t *status) {
-  volatile uint32_t *cell = &ctrl.fifo[head];
-  uint32_t word = *cell;
-  if (word == 0) {
-    const long long start = clock64();
-    uint32_t n = 0;
-    while ((word = *cell) == 0) {
-      if ((++n & 63u) == 0) {
-        if (*reinterpret_cast<volatile int *>(&ctrl.abort)) return kCmdExit;
-        if (clock64() - start > ctrl.timeout_cycles) {
-          *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
-          atomicExch(status, 5);
-          return kCmdExit;
-        }
-      }
-    }
-  }
-  *cell = 0;
-  head = (head + 1) & (kFifoDepth - 1);
-  return word;
-}
-
 // The producer is also the scheduler: it walks the items, issues the TMA loads and publishes one
 // command word per slot-step (PV(s, t) fused with the S(s, t + 1) that follows it), so the MMA
 // issuer's own loop stays a few instructions long.
@@ -260,8 +244,16 @@ template <int D>
 __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, const CUtensorMap *map_k,
                               const CUtensorMap *map_v, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring) {
   using C = Cfg<D>;
+  // measurement hook: the SM clock this CTA really ran at is cycles / nanoseconds over its run
+  const bool probe = p.clock_probe != nullptr && blockIdx.x == 0;
+  long long probe_c0 = 0;
+  unsigned long long probe_t0 = 0;
+  if (probe) {
+    probe_c0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(probe_t0));
+  }
   RingPos ring{0, 0};
-  uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, fills = 0, tail = 0, pending = 0;
+  uint32_t n_use0 = 0, n_use1 = 0, n_sp0 = 0, n_sp1 = 0, n_s = 0, fills = 0, tail = 0, pending = 0;
   bool ok = true;
   const bool stalled = p.stall_cta == int(blockIdx.x);
   const int k_end = p.cta_begin[blockIdx.x + 1];
@@ -296,34 +288,41 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
       // phase of this item's use of the slot: Q-full for S, O-empty (inverted) for PV
       const uint32_t use_phase = ((s ? n_use1 : n_use0) - 1u) & 1u;
       if (is_s) {
+        // the S buffer is shared: S number n may be issued once S number n - 1 has been loaded into registers
         uint32_t part = kCmdHasS | (f.slot << kCmdKRingShift) | (f.phase ? kCmdKPhase : 0u) |
-                        (first ? 0u : kCmdKSkipWait) | (final_use ? kCmdKFinal : 0u);
+                        (first ? 0u : kCmdKSkipWait) | (final_use ? kCmdKFinal : 0u) |
+                        (n_s > 0 ? kCmdWaitSFree : 0u) | (((n_s - 1u) & 1u) ? kCmdSFreePhase : 0u);
+        ++n_s;
         if (t == w.lo(s)) part |= kCmdWaitQFull | (use_phase ? kCmdQFullPhase : 0u);
         if (t == w.hi(s)) part |= kCmdQEnd;
-        // S(s, t) directly follows PV(s, t - 1) of the same slot: complete that command; otherwise
-        // (first step of the slot) it goes out alone
-        uint32_t cmd = pending | part | kCmdValid | (s ? kCmdSlot1 : 0u);
-        pending = 0;
-        if (stalled) return true;  // test hook: the issuer's bounded wait for this command must expire
-        return fifo_push(ctrl, tail, cmd, p.status);
+        if (t == w.lo(s)) {
+          // first step of the slot: nothing of this slot to pair it with
+          if (stalled) return true;  // test hook: the issuer's bounded wait for this command must expire
+          return fifo_push(ctrl, tail, part | kCmdValid | (s ? kCmdSlot1 : 0u), p.status);
+        }
+        pending = part;  // completed by the PV(s, t - 1) that the walk visits next
+        return true;
       }
       uint32_t &n_sp = s ? n_sp1 : n_sp0;
       uint32_t part = kCmdHasPV | (f.slot << kCmdVRingShift) | (f.phase ? kCmdVPhase : 0u) |
                       (first ? 0u : kCmdVSkipWait) | (final_use ? kCmdVFinal : 0u) | (t > w.lo(s) ? kCmdAcc : 0u) |
                       ((n_sp & 1u) ? kCmdPPhase : 0u);
       if (t == w.lo(s)) part |= kCmdWaitOEmpty | ((use_phase ^ 1u) ? kCmdOEmptyPhase : 0u);
+      if (t == w.hi(s)) part |= kCmdOEnd;
       ++n_sp;
-      if (t == w.hi(s)) {
-        // last step of the slot: no S follows
-        const uint32_t cmd = part | kCmdOEnd | kCmdValid | (s ? kCmdSlot1 : 0u);
-        if (stalled) return true;
-        return fifo_push(ctrl, tail, cmd, p.status);
-      }
-      pending = part;  // completed by the S(s, t + 1) that the walk visits next
-      return true;
+      const uint32_t cmd = pending | part | kCmdValid | (s ? kCmdSlot1 : 0u);
+      pending = 0;
+      if (stalled) return true;
+      return fifo_push(ctrl, tail, cmd, p.status);
     });
   }
   if (ok) ok = fifo_push(ctrl, tail, kCmdValid | kCmdExit, p.status);
+  if (probe) {
+    unsigned long long t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    p.clock_probe[0] = clock64() - probe_c0;
+    p.clock_probe[1] = (long long)(t1 - probe_t0);
+  }
   if (!ok) {
     // leave only after the copies already issued have landed (bounded), so none writes into
     // shared memory of a later CTA: the last min(fills, stages) fills end at ring.slot - 1
@@ -352,78 +351,148 @@ __device__ void producer_role(const KernelParams &p, const CUtensorMap *map_q, c
 }
 
 // ------------------------------------------------------------------------------------------------
+// tcgen05.mma, tcgen05.commit and mbarrier tests take their operands from the warp's uniform
+// registers, so the issuing warp keeps everything it derives from a command word provably uniform:
+// all 32 lanes run the loop and read the same queue cell, and the word is rebuilt by a warp vote
+// (lane i contributes bit i).  A value loaded from shared memory by one lane is not uniform as far
+// as the compiler can tell, and every operand derived from it would be copied into a uniform
+// register again before each instruction that needs it.
+__device__ __forceinline__ uint32_t warp_uniform(uint32_t word, int lane) {
+  return __ballot_sync(0xffffffffu, (word >> lane) & 1u);
+}
+
+// Pop by the whole warp: every lane polls the same cell; the decision to leave is taken on the
+// voted word, so the lanes stay together.  Lane 0 empties the cell.
+__device__ __forceinline__ uint32_t fifo_pop_warp(Ctrl &ctrl, uint32_t &head, int32_t *status, int lane) {
+  volatile uint32_t *cell = &ctrl.fifo[head];
+  __syncwarp();
+  uint32_t word = warp_uniform(*cell, lane);
+  if (word == 0) {
+    const long long start = clock64();
+    uint32_t n = 0;
+    while (true) {
+      __syncwarp();
+      word = warp_uniform(*cell, lane);
+      if (word != 0) break;
+      if ((++n & 63u) == 0) {
+        const bool stop = *reinterpret_cast<volatile int *>(&ctrl.abort) != 0 || clock64() - start > ctrl.timeout_cycles;
+        if (__any_sync(0xffffffffu, stop)) {
+          if (lane == 0 && *reinterpret_cast<volatile int *>(&ctrl.abort) == 0) {
+            *reinterpret_cast<volatile int *>(&ctrl.abort) = 1;
+            atomicExch(status, 5);
+          }
+          return kCmdExit;
+        }
+      }
+    }
+  }
+  if (lane == 0) *cell = 0;
+  head = (head + 1) & (kFifoDepth - 1);
+  return word;
+}
+
 template <int D>
-__device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring) {
+__device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uint8_t *smem_ring, const int lane) {
   using C = Cfg<D>;
-  const uint32_t tmem = ctrl.tmem_base;
+  const uint32_t tmem = warp_uniform(ctrl.tmem_base, lane);
   const uint32_t idesc_s = make_idesc_bf16(kTile, kTile, 0, 0);
   const uint32_t idesc_pv = make_idesc_bf16(kTile, D, 0, 1);
-  // K-major operands (Q, K): 8-row groups 1024 bytes apart.  V is MN-major: 8-key groups 1024
-  // bytes apart, the next 64 columns of head_dim one box further.
   const uint64_t desc_q0 = make_smem_desc(smem_u32(smem_q), 16, 1024);
   const uint64_t desc_k0 = make_smem_desc(smem_u32(smem_ring), 16, 1024);
   const uint64_t desc_v0 = make_smem_desc(smem_u32(smem_ring), C::kBoxBytes, 1024);
   uint32_t head = 0;
-  uint32_t cmd = fifo_pop(ctrl, head, p.status);
+  bool ok = true;
+  TRACE_DECL(8);
+#ifdef STEEL_TRACE
+  const long long role_t0 = clock64();
+#endif
+  uint32_t cmd = fifo_pop_warp(ctrl, head, p.status, lane);
   while (!(cmd & kCmdExit)) {
-    // look at the next command now, so that its shared-memory latency hides behind this one's issue
     volatile uint32_t *next_cell = &ctrl.fifo[head];
-    const uint32_t next = *next_cell;
+    __syncwarp();
+    const uint32_t next_raw = *next_cell;
     const uint32_t s = (cmd & kCmdSlot1) ? 1u : 0u;
-    const uint32_t t_s = tmem + C::kColS + s * kTile;
     const uint32_t v_slot = (cmd >> kCmdVRingShift) & 0xFu, k_slot = (cmd >> kCmdKRingShift) & 0xFu;
     const bool has_pv = (cmd & kCmdHasPV) != 0, has_s = (cmd & kCmdHasS) != 0;
-    // test the barriers this command depends on back to back, so their latencies overlap; only the
-    // ones not yet complete are then waited for
-    const bool need_v = has_pv && !(cmd & kCmdVSkipWait), need_k = has_s && !(cmd & kCmdKSkipWait);
-    bool ok_v = !need_v || mbar_test_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u);
-    bool ok_k = !need_k || mbar_test_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u);
-    bool ok_p = !has_pv || mbar_test_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u);
-    // rare waits (first / last step of an item) and barriers that were not yet complete
     constexpr uint32_t kRare = kCmdWaitOEmpty | kCmdWaitQFull | kCmdOEnd | kCmdQEnd;
     const uint32_t rare = cmd & kRare;
-    if (rare | uint32_t(!ok_v) | uint32_t(!ok_k) | uint32_t(!ok_p)) {
-      bool ok = true;
-      if (cmd & kCmdWaitOEmpty) ok = bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status);
-      if (ok && (cmd & kCmdWaitQFull))
-        ok = bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status);
-      if (ok && !ok_v) ok = bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status);
-      if (ok && !ok_k) ok = bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status);
-      if (ok && !ok_p) ok = bounded_wait(&ctrl.p_full[s], (cmd & kCmdPPhase) ? 1u : 0u, ctrl, p.status);
-      if (!ok) break;
-    }
-    tc_fence_after();
-    if (has_pv) {
-      const uint64_t dv = desc_v0 + uint64_t((v_slot * C::kTileBytes) >> 4);
-      const uint32_t t_o = tmem + C::kColO + s * D;
-      const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u;
+    if (elect_one()) {
+      TRACE_T0();
+      const bool need_v = has_pv && !(cmd & kCmdVSkipWait), need_k = has_s && !(cmd & kCmdKSkipWait);
+      const bool need_f = has_s && (cmd & kCmdWaitSFree);
+      uint64_t *s_free = &ctrl.s_free;
+      bool ok_f = !need_f || mbar_test_wait(s_free, (cmd & kCmdSFreePhase) ? 1u : 0u);
+      bool ok_k = !need_k || mbar_test_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u);
+      bool ok_v = !need_v || mbar_test_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u);
+      if (has_s) {
+        if (rare | uint32_t(!ok_f) | uint32_t(!ok_k)) {
+          if (cmd & kCmdWaitQFull)
+            ok = bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status);
+          if (ok && !ok_f) { TRACE_T0(); ok = bounded_wait(s_free, (cmd & kCmdSFreePhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(0); }
+          if (ok && !ok_k) { TRACE_T0(); ok = bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(1); }
+        }
+        if (ok) {
+          tc_fence_after();
+          const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
+          const uint64_t dk = desc_k0 + uint64_t((k_slot * C::kTileBytes) >> 4);
 #pragma unroll
-      for (int kk = 0; kk < kTile / 16; ++kk)
-        mma_ts(t_o, t_s + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
-      tc_commit_if(&ctrl.ring_empty[v_slot], cmd & kCmdVFinal);
-    }
-    if (has_s) {
-      const uint64_t dq = desc_q0 + uint64_t((s * C::kTileBytes) >> 4);
-      const uint64_t dk = desc_k0 + uint64_t((k_slot * C::kTileBytes) >> 4);
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
-        mma_ss(t_s, dq + off, dk + off, idesc_s, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
+            mma_ss(tmem + C::kColS, dq + off, dk + off, idesc_s, kk > 0);
+          }
+          tc_commit(&ctrl.s_full[s]);
+          tc_commit_if(&ctrl.ring_empty[k_slot], cmd & kCmdKFinal);
+          if (rare) tc_commit_if(&ctrl.q_empty[s], cmd & kCmdQEnd);
+        }
       }
-      tc_commit(&ctrl.s_full[s]);
-      tc_commit_if(&ctrl.ring_empty[k_slot], cmd & kCmdKFinal);
+      if (ok && has_pv) {
+        const uint32_t p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
+        const bool ok_p = mbar_test_wait(&ctrl.p_full[s], p_phase);
+        if (rare | uint32_t(!ok_p) | uint32_t(!ok_v)) {
+          if (cmd & kCmdWaitOEmpty) ok = bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status);
+          if (ok && !ok_v) { TRACE_T0(); ok = bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(2); }
+          if (ok && !ok_p) { TRACE_T0(); ok = bounded_wait(&ctrl.p_full[s], p_phase, ctrl, p.status); TRACE_ADD(3); }
+        }
+        if (ok) {
+          tc_fence_after();
+          const uint64_t dv = desc_v0 + uint64_t((v_slot * C::kTileBytes) >> 4);
+          const uint32_t t_p = tmem + C::kColP + s * (kTile / 2);
+          const uint32_t t_o = tmem + C::kColO + s * D;
+          const uint32_t acc0 = (cmd & kCmdAcc) ? 1u : 0u;
+#pragma unroll
+          for (int kk = 0; kk < kTile / 16; ++kk)
+            mma_ts(t_o, t_p + kk * 8, dv + uint64_t((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+          tc_commit(&ctrl.p_free[s]);
+          tc_commit_if(&ctrl.ring_empty[v_slot], cmd & kCmdVFinal);
+          if (rare) tc_commit_if(&ctrl.o_full[s], cmd & kCmdOEnd);
+        }
+      }
+      TRACE_ADD(5);
     }
-    if (rare) {
-      // all of this command's MMAs are issued: these commits cover them
-      tc_commit_if(&ctrl.o_full[s], cmd & kCmdOEnd);
-      tc_commit_if(&ctrl.q_empty[s], cmd & kCmdQEnd);
-    }
+    const uint32_t next = warp_uniform(next_raw, lane);
+    if (__any_sync(0xffffffffu, !ok)) break;
     if (next != 0) {
-      *next_cell = 0;
+      if (lane == 0) *next_cell = 0;
       head = (head + 1) & (kFifoDepth - 1);
       cmd = next;
     } else {
-      cmd = fifo_pop(ctrl, head, p.status);
+      TRACE_T0();
+      cmd = fifo_pop_warp(ctrl, head, p.status, lane);
+      TRACE_ADD(4);
+    }
+  }
+#ifdef STEEL_TRACE
+  trace_acc[7] = clock64() - role_t0;
+  if (elect_one()) { TRACE_FLUSH(0, 8); }
+#endif
+  // Leaving on an expired wait: everything this warp issued must have retired before the CTA frees
+  // its tensor memory, so commit to a spare barrier and wait for it (bounded).
+  if (*reinterpret_cast<volatile int *>(&ctrl.abort)) {
+    if (elect_one()) {
+      tc_commit(&ctrl.drain);
+      const long long start = clock64();
+      while (!mbar_try_wait(&ctrl.drain, 0) && clock64() - start < ctrl.timeout_cycles / 8) {
+      }
     }
   }
 }
@@ -448,7 +517,9 @@ __device__ __forceinline__ float2 exp2_poly(float2 y) {
 }
 
 // exp2 of 64 scaled scores -> 32 packed bf16x2 registers; accumulates the row sum in two lane pairs.
-// With kEmu > 0, one pair in every 2^(3 - kEmu) is evaluated by exp2_poly (12.5 %, 25 %, 50 %).
+// With kEmu > 0, one pair in every 2^(3 - kEmu) is evaluated by exp2_poly (12.5 %, 25 %, 50 % of the
+// exponentials leave the special-function unit for the FMA pipe: the counterpart of the lookup-table
+// exponent the paper uses on the NPU generation that has no exponent unit).
 template <int kEmu>
 __device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, float2 scale2, float2 neg_m2,
                                          float2 &acc_a, float2 &acc_b, uint32_t (&packed)[32]) {
@@ -473,12 +544,13 @@ __device__ __forceinline__ void exp_half(const float (&x)[kTile], int base, floa
   }
 }
 
-template <int D>
+template <int D, int kEmu>
 __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, const int r) {
   using C = Cfg<D>;
   const int lane = r % 32;
   const uint32_t lane_base = uint32_t((r / 32) * 32) << 16;
-  const uint32_t t_s = ctrl.tmem_base + lane_base + C::kColS + s * kTile;
+  const uint32_t t_s = ctrl.tmem_base + lane_base + C::kColS;
+  const uint32_t t_p = ctrl.tmem_base + lane_base + C::kColP + s * (kTile / 2);
   const uint32_t t_o = ctrl.tmem_base + lane_base + C::kColO + s * D;
   const bool causal = (p.mask_flags & kMaskCausal) != 0, windowed = (p.mask_flags & kMaskWindow) != 0;
   const int off = p.seq_kv - p.seq_q;
@@ -489,6 +561,8 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
   TRACE_DECL(7);
 #ifdef STEEL_TRACE
   const long long role_t0 = clock64();
+  unsigned long long gt0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
 #endif
 
   const int k_end = p.cta_begin[blockIdx.x + 1];
@@ -540,6 +614,10 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         for (int i = 0; i < 32; ++i) x[c * 32 + i] = __uint_as_float(regs[i]);
       }
       tc_wait_ld();
+      // the scores are in registers: hand the S buffer back for the next QK^T (of either slot)
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl.s_free);
       TRACE_ADD(2);
 
       if (partial) {
@@ -574,6 +652,9 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
         // the running maximum only has to bound the exponents: rescale O lazily
         const bool need = ms > m_ref + kRescaleThreshold;
         if (__any_sync(0xffffffffu, need)) {
+          // PV(s, t - 1) accumulates into O: it must have finished
+          if (!warp_wait(&ctrl.p_free[s], (n_sp - 1u) & 1u, ctrl, p.status, lane)) return;
+          tc_fence_after();
           const float v = need ? ex2_approx(m_ref - ms) : 1.0f;
           l *= v;
 #pragma unroll
@@ -595,10 +676,14 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t packed[32];
-        // masked (-inf) scores keep the exact special-function path so that empty rows sum to 0
-        if (kExpEmulation == 0 || partial) exp_half<0>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
-        else exp_half<kExpEmulation>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
-        tmem_st32(t_s + half * 32, packed);
+        exp_half<kEmu>(x, half * 64, scale2, neg_m2, acc_a, acc_b, packed);
+        if (half == 0 && t > lo) {
+          // PV(s, t - 1) reads the P columns: it must have finished before they are overwritten (by
+          // now it has had the whole first half of the exponentials to do so)
+          if (!warp_wait(&ctrl.p_free[s], (n_sp - 1u) & 1u, ctrl, p.status, lane)) return;
+          tc_fence_after();
+        }
+        tmem_st32(t_p + half * 32, packed);
       }
       tc_wait_st();
       tc_fence_before();
@@ -606,7 +691,9 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
       if (lane == 0) mbar_arrive(&ctrl.p_full[s]);
       ++n_sp;
       const float2 acc = fadd2(acc_a, acc_b);
-      l += acc.x + acc.y;
+      // The polynomial path returns 2^-125 rather than 0 for a masked (-inf) score: a row that has
+      // not seen a visible key yet (m = -inf) must keep l = 0 exactly, so that it ends as O = 0.
+      if (kEmu == 0 || m_ref != -CUDART_INF_F) l += acc.x + acc.y;
       TRACE_ADD(3);
     }
 
@@ -658,13 +745,16 @@ __device__ void softmax_role(const KernelParams &p, Ctrl &ctrl, const int s, con
 #ifdef STEEL_TRACE
   trace_acc[6] = clock64() - role_t0;
   if (r == 0) {
+    unsigned long long gt1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
+    if (p.trace && s == 0) p.trace[size_t(blockIdx.x) * 32 + 15] = (long long)(gt1 - gt0);
     TRACE_FLUSH(16 + 8 * s, 7);
   }
 #endif
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, int kEmu>
 __global__ void __launch_bounds__(kThreads, 1)
 steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ KernelParams p) {
@@ -686,9 +776,12 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(&ctrl.q_empty[s], 1);
       mbar_init(&ctrl.s_full[s], 1);
       mbar_init(&ctrl.p_full[s], 4);  // one arrival per softmax warp
+      mbar_init(&ctrl.p_free[s], 1);
       mbar_init(&ctrl.o_full[s], 1);
       mbar_init(&ctrl.o_empty[s], 4);
     }
+    mbar_init(&ctrl.s_free, 4);
+    mbar_init(&ctrl.drain, 1);
     for (int i = 0; i < kFifoDepth; ++i) ctrl.fifo[i] = 0;
     ctrl.abort = 0;
     ctrl.timeout_cycles = p.timeout_cycles;
@@ -709,13 +802,13 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
   if (warp < 8) {
     setmaxnreg_inc<kRegsSoftmax>();
-    softmax_role<D>(p, ctrl, warp / 4, threadIdx.x % kTile);
+    softmax_role<D, kEmu>(p, ctrl, warp / 4, threadIdx.x % kTile);
   } else {
     setmaxnreg_dec<kRegsOther>();
     if (warp == kProducerWarp) {
       if (lane == 0) producer_role<D>(p, &map_q, &map_k, &map_v, ctrl, smem_q, smem_ring);
     } else if (warp == kMmaWarp) {
-      if (lane == 0) mma_role<D>(p, ctrl, smem_q, smem_ring);
+      mma_role<D>(p, ctrl, smem_q, smem_ring, lane);
     }
   }
 
@@ -725,20 +818,52 @@ steel_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   if (warp == kMmaWarp) tmem_dealloc(ctrl.tmem_base, 512);
 }
 
-cudaError_t configure_kernels() {
-  cudaError_t e = cudaFuncSetAttribute(steel_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       Cfg<128>::kSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(steel_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<64>::kSmemBytes);
+namespace {
+
+template <int D, int kEmu>
+cudaError_t configure_one() {
+  return cudaFuncSetAttribute(steel_attn_kernel<D, kEmu>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<D>::kSmemBytes);
 }
 
-cudaError_t launch_attention(int head_dim, const CUtensorMap &map_q, const CUtensorMap &map_k,
+template <int D, int kEmu>
+void launch_one(const CUtensorMap &map_q, const CUtensorMap &map_k, const CUtensorMap &map_v,
+                const KernelParams &params, int grid, cudaStream_t stream) {
+  steel_attn_kernel<D, kEmu><<<grid, kThreads, Cfg<D>::kSmemBytes, stream>>>(map_q, map_k, map_v, params);
+}
+
+template <int D>
+void launch_dim(int exp_emulation, const CUtensorMap &map_q, const CUtensorMap &map_k, const CUtensorMap &map_v,
+                const KernelParams &params, int grid, cudaStream_t stream) {
+  switch (exp_emulation) {
+    case 1: launch_one<D, 1>(map_q, map_k, map_v, params, grid, stream); break;
+    case 2: launch_one<D, 2>(map_q, map_k, map_v, params, grid, stream); break;
+    case 3: launch_one<D, 3>(map_q, map_k, map_v, params, grid, stream); break;
+    default: launch_one<D, 0>(map_q, map_k, map_v, params, grid, stream); break;
+  }
+}
+
+}  // namespace
+
+cudaError_t configure_kernels() {
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = configure_one<128, 0>();
+  if (e == cudaSuccess) e = configure_one<128, 1>();
+  if (e == cudaSuccess) e = configure_one<128, 2>();
+  if (e == cudaSuccess) e = configure_one<128, 3>();
+  if (e == cudaSuccess) e = configure_one<64, 0>();
+  if (e == cudaSuccess) e = configure_one<64, 1>();
+  if (e == cudaSuccess) e = configure_one<64, 2>();
+  if (e == cudaSuccess) e = configure_one<64, 3>();
+  return e;
+}
+
+cudaError_t launch_attention(int head_dim, int exp_emulation, const CUtensorMap &map_q, const CUtensorMap &map_k,
                              const CUtensorMap &map_v, const KernelParams &params, int grid, cudaStream_t stream) {
   if (head_dim == 128)
-    steel_attn_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(map_q, map_k, map_v, params);
+    launch_dim<128>(exp_emulation, map_q, map_k, map_v, params, grid, stream);
   else
-    steel_attn_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(map_q, map_k, map_v, params);
+    launch_dim<64>(exp_emulation, map_q, map_k, map_v, params, grid, stream);
   return cudaGetLastError();
 }
 

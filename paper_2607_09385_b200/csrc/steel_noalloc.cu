@@ -84,7 +84,7 @@ extern "C" steel_status_t steel_attn_run_noalloc(const steel_attn_params_t *para
 
   Plan plan;  // host memory only
   try {
-    st = build_plan(params, sm_count, 0, &plan);
+    st = build_plan(params, sm_count, &plan, /*exec_stats=*/false);
   } catch (const std::bad_alloc &) {
     return STEEL_ERR_ALLOC;
   }
@@ -114,9 +114,10 @@ extern "C" steel_status_t steel_attn_run_noalloc(const steel_attn_params_t *para
   kp.steps = reinterpret_cast<const StepPair *>(base + kOffSteps);
   kp.status = reinterpret_cast<int32_t *>(base + kOffStatus);
   kp.trace = nullptr;
+  kp.clock_probe = nullptr;
   kp.timeout_cycles = kDefaultTimeoutCycles;
   kp.stall_cta = -1;
-  st = launch_with_params(*params, kp, plan.grid, q, k, v, o, lse, stream);
+  st = launch_with_params(*params, kp, plan.grid, q, k, v, o, lse, stream, nullptr);
   if (st != STEEL_OK) return st;
   // Blocking by design: the host lists above must outlive the copies, and the status word has to
   // be read before the next call clears it.

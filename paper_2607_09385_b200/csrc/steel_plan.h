@@ -54,6 +54,7 @@ struct KernelParams {
   int32_t window;            // clamped to int32 range
   float scale_log2;          // scale * log2(e)
   long long *trace;          // per-CTA wait accounting (debug builds only), else null
+  long long *clock_probe;    // measurement hook: CTA 0 stores {SM cycles, nanoseconds} of its run here, else null
   long long timeout_cycles;  // bound of every device-side wait
   int32_t stall_cta;         // test hook: this CTA's producer withholds its commands (-1: none)
 };

@@ -119,6 +119,7 @@ steel_status_t validate_params(const steel_attn_params_t *p) {
   if ((p->mask.flags & STEEL_MASK_WINDOW) && p->mask.window <= 0) return STEEL_ERR_INVALID_ARG;
   if ((p->mask.flags & STEEL_MASK_BITMAP) && !p->mask.bitmap) return STEEL_ERR_INVALID_ARG;
   if (p->mask.block_q < 0 || p->mask.block_kv < 0) return STEEL_ERR_INVALID_ARG;
+  if (p->policy < 0 || p->policy > 2 || p->exp_emulation < 0 || p->exp_emulation > 3) return STEEL_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return STEEL_ERR_UNSUPPORTED;
   int bq = p->mask.block_q ? p->mask.block_q : kTile, bkv = p->mask.block_kv ? p->mask.block_kv : kTile;
   if (bq != bkv || (bq != 64 && bq != 128)) return STEEL_ERR_UNSUPPORTED;
@@ -129,9 +130,10 @@ steel_status_t validate_params(const steel_attn_params_t *p) {
   return STEEL_OK;
 }
 
-steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy, Plan *plan) {
+steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, Plan *plan, bool exec_stats) {
   steel_status_t st = validate_params(p);
   if (st != STEEL_OK) return st;
+  const int policy = p->policy;
   if (num_ctas <= 0 || !plan) return STEEL_ERR_INVALID_ARG;
 
   Ctx c;
@@ -450,7 +452,8 @@ steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy
     for (int id : per_cta[cta]) st_sum += drafts[id].w.n_steps;
     s.max_cta_steps = std::max(s.max_cta_steps, st_sum);
   }
-  walk_plan(*plan, [&](int, const WorkItem &, int, int, uint32_t entry, bool shared) {
+  // the walk visits every executed tile (millions on long sequences): only for callers that read these
+  if (exec_stats) walk_plan(*plan, [&](int, const WorkItem &, int, int, uint32_t entry, bool shared) {
     ++s.exec_tiles;
     s.exec_partial += (entry & kEntryPartial) != 0;
     s.kv_tile_loads += shared ? 0 : 1;

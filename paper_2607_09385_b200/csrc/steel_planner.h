@@ -27,7 +27,9 @@ struct Plan {
 };
 
 steel_status_t validate_params(const steel_attn_params_t *p);
-steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, int policy, Plan *plan);
+// Scheduling policy and the other options come from `p`.  `exec_stats` = false skips the statistics
+// that need a walk over every executed tile (exec_tiles, exec_partial, kv_tile_loads stay 0).
+steel_status_t build_plan(const steel_attn_params_t *p, int num_ctas, Plan *plan, bool exec_stats = true);
 
 // Entry (tile index and flags, 0 if absent) of `slot` at step `t`, derived exactly as on the device.
 uint32_t item_entry(const Plan &plan, const WorkItem &w, int slot, int t, const steel_attn_params_t *p);

@@ -12,9 +12,10 @@ def to_device(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def make_attention(w: inputs.Workload, bitmap=None, scale=None) -> binding.SteelAttention:
+def make_attention(w: inputs.Workload, bitmap=None, scale=None, policy=0, exp_emulation=0) -> binding.SteelAttention:
     return binding.SteelAttention(w.batch, w.heads_q, w.heads_kv, w.seq, w.seq, w.head_dim,
-                                  w.scale if scale is None else scale, w.flags, w.block, w.window, bitmap)
+                                  w.scale if scale is None else scale, w.flags, w.block, w.window, bitmap,
+                                  policy=policy, exp_emulation=exp_emulation)
 
 
 def oracle_problem(w: inputs.Workload, bitmap=None, scale=None) -> oracle.OracleProblem:
@@ -22,9 +23,9 @@ def oracle_problem(w: inputs.Workload, bitmap=None, scale=None) -> oracle.Oracle
                                 w.scale if scale is None else scale, w.flags, w.block, w.block, w.window, bitmap)
 
 
-def run_gpu(w, data, scale=None, poison=True):
+def run_gpu(w, data, scale=None, poison=True, policy=0, exp_emulation=0):
     """Run the CUDA path on workload `w`; outputs are pre-filled with NaN so unwritten rows show."""
-    attn = make_attention(w, data["bitmap"], scale)
+    attn = make_attention(w, data["bitmap"], scale, policy, exp_emulation)
     q, k, v = (to_device(data[x]) for x in "qkv")
     o = torch.full_like(q, float("nan")) if poison else torch.empty_like(q)
     lse = torch.full((w.batch, w.heads_q, w.seq), float("nan"), dtype=torch.float32, device="cuda")

@@ -25,7 +25,7 @@ def test_library_exports_every_declared_symbol(repo_root):
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(B.MaskDesc) == 32 and ctypes.sizeof(B.Params) == 64
+    assert ctypes.sizeof(B.MaskDesc) == 32 and ctypes.sizeof(B.Params) == 72
     assert ctypes.sizeof(B.Stats) == 13 * 8
 
 
@@ -60,7 +60,10 @@ def test_validation_codes():
     assert lib.steel_attn_plan_host(None, ctypes.byref(B.Stats()), None, 0, None) == B.STEEL_ERR_INVALID_ARG
     assert lib.steel_attn_destroy(None) == B.STEEL_OK
     assert lib.steel_attn_get_stats(None, None) == B.STEEL_ERR_INVALID_ARG
-    assert lib.steel_attn_set_policy(7) == B.STEEL_ERR_INVALID_ARG
+    assert plan(policy=7) == B.STEEL_ERR_INVALID_ARG
+    assert plan(policy=-1) == B.STEEL_ERR_INVALID_ARG
+    assert plan(exp_emulation=4) == B.STEEL_ERR_INVALID_ARG
+    assert plan(exp_emulation=3, policy=2) == B.STEEL_OK
     assert lib.steel_attn_create(None, None) == B.STEEL_ERR_INVALID_ARG
 
 

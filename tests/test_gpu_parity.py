@@ -68,6 +68,9 @@ EDGE_CASES = [
     dict(name="window_unaligned", B=1, Hq=2, Hkv=2, S=1024, D=128, flags=CAUSAL | WINDOW, window=300),
     dict(name="window_tiny", B=1, Hq=1, Hkv=1, S=512, D=64, flags=CAUSAL | WINDOW, window=1),
     dict(name="window_only", B=1, Hq=2, Hkv=2, S=768, D=128, flags=WINDOW, window=200),
+    # a window far beyond 32 bits hides nothing; with a ragged last key tile the kernel's column
+    # arithmetic must not overflow
+    dict(name="window_huge_ragged", B=1, Hq=2, Hkv=1, S=1000, D=128, flags=WINDOW, window=1 << 40),
     dict(name="bitmap128", B=1, Hq=4, Hkv=4, S=2048, D=128, flags=CAUSAL | BITMAP, keep=0.3),
     dict(name="bitmap64_d64", B=1, Hq=2, Hkv=2, S=1024, D=64, flags=CAUSAL | BITMAP, block=64, keep=0.4),
     dict(name="bitmap_gqa", B=2, Hq=4, Hkv=2, S=1024, D=128, flags=CAUSAL | BITMAP, keep=0.5),
@@ -194,11 +197,7 @@ def test_other_placement_policies_match(policy):
     w = inputs.Workload("policy", 1, 4, 4, 2048, 128, 128, CAUSAL)
     data = inputs.make_inputs(w, seed=31)
     attn0, o0, lse0 = H.run_gpu(w, data)
-    binding.steel_attn_set_policy(policy)
-    try:
-        attn1, o1, lse1 = H.run_gpu(w, data)
-    finally:
-        binding.steel_attn_set_policy(0)
+    attn1, o1, lse1 = H.run_gpu(w, data, policy=policy)
     H.assert_parity(w, data, o1, lse1, H.sampled_rows(w, range(4), 1, 64))
     assert (o0.float() - o1.float()).abs().max() <= 2e-2
     attn0.close()

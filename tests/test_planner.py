@@ -13,8 +13,8 @@ from paper_2607_09385_b200 import inputs
 CAUSAL, WINDOW, BITMAP = inputs.MASK_CAUSAL, inputs.MASK_WINDOW, inputs.MASK_BITMAP
 
 
-def host_plan(batch, hq, hkv, sq, skv, d, flags, block=128, window=0, bitmap=None, tiles=True):
-    p, keep = B.make_params(batch, hq, hkv, sq, skv, d, 0.1, flags, block, block, window, bitmap)
+def host_plan(batch, hq, hkv, sq, skv, d, flags, block=128, window=0, bitmap=None, tiles=True, policy=0):
+    p, keep = B.make_params(batch, hq, hkv, sq, skv, d, 0.1, flags, block, block, window, bitmap, policy)
     st, stats, recs = B.steel_attn_plan_host(p, want_tiles=tiles)
     assert st == B.STEEL_OK
     return stats, recs
@@ -150,17 +150,14 @@ def test_balance_and_policies():
     key = lambda r: {tuple(x[1:5]) for x in r}
     by_policy = {0: stats}
     for policy in (1, 2):
-        B.steel_attn_set_policy(policy)
-        try:
-            by_policy[policy], recs = host_plan(1, w.heads_q, w.heads_kv, w.seq, w.seq, 128, w.flags, tiles=True)
-        finally:
-            B.steel_attn_set_policy(0)
+        by_policy[policy], recs = host_plan(1, w.heads_q, w.heads_kv, w.seq, w.seq, 128, w.flags, tiles=True,
+                                            policy=policy)
         assert key(recs0) == key(recs) and by_policy[policy]["exec_tiles"] == stats["exec_tiles"]
     # contiguous chunks (uniform placement) are the most unbalanced under a causal mask, dealing
     # consecutive tiles round-robin (sparsity-aware placement) is better, longest-first is best
     assert by_policy[1]["max_cta_steps"] > by_policy[2]["max_cta_steps"] > by_policy[0]["max_cta_steps"]
-    lib = B.load_library()
-    assert lib.steel_attn_set_policy(3) == B.STEEL_ERR_INVALID_ARG
+    bad, _ = B.make_params(1, 2, 2, 256, 256, 128, 0.1, w.flags, policy=3)
+    assert B.steel_attn_plan_host(bad)[0] == B.STEEL_ERR_INVALID_ARG
 
 
 def test_makespan_model_of_uniform_vs_interleaved_placement():
