@@ -34,10 +34,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL_BF16_TFLOPS = 2250.0  # vendor figure for dense bf16 on one B200 (context, not a measurement)
 # dram__bytes_read.sum + dram__bytes_write.sum of one kernel launch on the default workload,
 # from the ncu capture summarised in profiles/ (None until a capture exists for a workload).
-NCU_TRAFFIC_BYTES = {"c2_causal_s4k_mha32": 143.90e6 + 12.46e6,                 # one-pass captures of a full launch
-                     "c3_window4k_s16k_gqa32x8": 213.86e6 + 98.80e6,
-                     "c4_bitmap25_s32k_h16": 4 * (141.451008e6 + 16.546048e6),  # 4 x the 4-head capture
-                     "c5_causal_s128k_gqa32x8": 3.38e9 + 1.08e9}              # one-pass capture of a full launch
+NCU_TRAFFIC_BYTES = {"c2_causal_s4k_mha32": 100930304 + 11335936,          # one-pass captures of one full launch each
+                     "c3_window4k_s16k_gqa32x8": 213756928 + 99447296,
+                     "c4_bitmap25_s32k_h16": 408786176 + 118737408,
+                     "c5_causal_s128k_gqa32x8": 3695049472 + 1193544192}
 
 
 def load_peaks():
