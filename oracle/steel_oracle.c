@@ -9,11 +9,12 @@
  *                           dense mask row M (0 where a key is visible, -inf elsewhere):
  *                           O_i = softmax(scale * q_i K^T + M_i) V, LSE_i = ln sum_j
  *                           exp(scale * q_i.k_j + M_ij).  `scale` generalises 1/sqrt(d).
- *   steel_oracle_alg1_block Algorithm 1 of the paper (First / Second / Third Stage) for one
- *                           query block, in the paper's order and notation, executing only
- *                           the tiles that are not fully masked (Sec. "The STEEL Pipeline",
- *                           the three mask cases).  Used to pin that skipping tiles gives
- *                           the dense masked result.
+ *   steel_oracle_alg1_block the streaming form that Algorithm 1 of the paper describes, for one
+ *                           query block: each row carries a running maximum, a running sum
+ *                           and a rescaled accumulator through the key blocks, and only
+ *                           blocks that are not fully masked are visited (Sec. "The STEEL
+ *                           Pipeline", the three mask cases).  Used to pin that skipping
+ *                           tiles gives the dense masked result.
  *   steel_oracle_classify   the three mask cases for one tile, by brute force over every
  *                           (query, key) pair of the tile.
  *
@@ -163,13 +164,16 @@ void steel_oracle_rows(const oracle_problem_t *p, const uint16_t *q, const uint1
 }
 
 /*
- * Algorithm 1 for query block I of (b, h): the three procedures run one after another for
- * each key block j, in the paper's notation (A_ij, m, m', P_ij, v, l, O_i).  Readings of the
- * listing: m` is m'; l' = v*l + rowsum(P) and is committed with m <- m'; the Third Stage
- * accumulates (O <- v*O + P V); initial state m = -inf, l = 0, O = 0; scores carry the
- * factor log2(e), so the exponent is taken base 2; a row whose running maximum is still
- * -inf contributes P = 0 and v = 1.  Fully masked tiles are skipped; others are masked
- * element-wise.  Outputs: o[B_q][d], lse[B_q] (natural log), returns the executed tiles.
+ * Tile-skipping streaming softmax for query block I of (b, h): the check that Algorithm 1 (tiles,
+ * running maximum, running sum, rescaled accumulator, skipped tiles) reproduces Eq. 1.  Written
+ * row by row: each query row carries its own state (top = largest score seen, mass = sum of
+ * 2^(score - top), acc = sum of 2^(score - top) * V) through the key blocks that the mask keeps.
+ * Readings of the paper used here: the new maximum replaces the old one after the sum is updated;
+ * the accumulator is rescaled and added to, not overwritten; the state starts at top = -inf,
+ * mass = 0, acc = 0; scores carry the factor log2(e) and the exponent is base 2; while a row has
+ * seen no visible key it adds nothing and rescales by 1.  A key block with no visible element for
+ * the whole query block is skipped; any other block is masked element by element.
+ * Outputs: o[B_q][d], lse[B_q] (natural log); returns the number of key blocks executed.
  */
 int64_t steel_oracle_alg1_block(const oracle_problem_t *p, const uint16_t *q,
                                 const uint16_t *k, const uint16_t *v, int b, int h, int I,
@@ -185,68 +189,60 @@ int64_t steel_oracle_alg1_block(const oracle_problem_t *p, const uint16_t *q,
   const int64_t i0 = (int64_t)I * bq;
   const int rows = (int)((i0 + bq <= sq) ? bq : sq - i0);
 
-  double *A = (double *)malloc(sizeof(double) * (size_t)bq * bkv);
-  double *P = (double *)malloc(sizeof(double) * (size_t)bq * bkv);
-  double *m = (double *)malloc(sizeof(double) * bq), *m_new = (double *)malloc(sizeof(double) * bq);
-  double *l = (double *)malloc(sizeof(double) * bq), *vv = (double *)malloc(sizeof(double) * bq);
-  for (int r = 0; r < rows; ++r) {
-    m[r] = -INFINITY;
-    l[r] = 0.0;
-    for (int c = 0; c < d; ++c) o[r * d + c] = 0.0;
-  }
+  /* which key blocks survive the skip rule, decided once for the whole query block */
+  unsigned char *keep = (unsigned char *)malloc((size_t)t_kv);
   int64_t executed = 0;
   for (int J = 0; J < t_kv; ++J) {
-    if (steel_oracle_classify(p, h, I, J) == 0) continue; /* case (i): skipped */
-    ++executed;
-    const int64_t j0 = (int64_t)J * bkv;
-    const int cols = (int)((j0 + bkv <= skv) ? bkv : skv - j0);
-    /* First Stage: A_ij = Q_i K_j^T, scale_and_mask, m' = max(m, rowmax(A_ij)) */
-    for (int r = 0; r < rows; ++r) {
-      double rowmax = -INFINITY;
+    keep[J] = steel_oracle_classify(p, h, I, J) != 0;
+    executed += keep[J];
+  }
+
+  double *score = (double *)malloc(sizeof(double) * (size_t)bkv);
+  for (int r = 0; r < rows; ++r) {
+    const int64_t i = i0 + r;
+    double *acc = o + (int64_t)r * d;
+    double top = -INFINITY, mass = 0.0;
+    for (int c = 0; c < d; ++c) acc[c] = 0.0;
+    for (int J = 0; J < t_kv; ++J) {
+      if (!keep[J]) continue;
+      const int64_t j0 = (int64_t)J * bkv;
+      const int cols = (int)((j0 + bkv <= skv) ? bkv : skv - j0);
+      /* scaled, masked scores of this row against the block, and their maximum */
+      double block_top = -INFINITY;
       for (int cj = 0; cj < cols; ++cj) {
         double s = 0.0;
         for (int c = 0; c < d; ++c)
-          s += bf16_to_f64(qbase[(i0 + r) * d + c]) * bf16_to_f64(kbase[(j0 + cj) * d + c]);
+          s += bf16_to_f64(qbase[i * d + c]) * bf16_to_f64(kbase[(j0 + cj) * d + c]);
         s *= p->scale * log2e;
-        if (!allowed(p, h, i0 + r, j0 + cj)) s = -INFINITY;
-        A[r * bkv + cj] = s;
-        if (s > rowmax) rowmax = s;
+        if (!allowed(p, h, i, j0 + cj)) s = -INFINITY;
+        score[cj] = s;
+        if (s > block_top) block_top = s;
       }
-      m_new[r] = rowmax > m[r] ? rowmax : m[r];
-    }
-    /* Second Stage: P = 2^(A - m'), v = 2^(m - m'), l <- v*l + rowsum(P), m <- m' */
-    for (int r = 0; r < rows; ++r) {
-      double rowsum = 0.0;
+      const double new_top = block_top > top ? block_top : top;
+      const int blind = new_top == -INFINITY; /* nothing visible so far */
+      /* move the state to the new maximum, then add this block's weights */
+      const double shrink = blind ? 1.0 : exp2(top - new_top);
+      double block_mass = 0.0;
+      for (int c = 0; c < d; ++c) acc[c] *= shrink;
       for (int cj = 0; cj < cols; ++cj) {
-        double pij = (m_new[r] == -INFINITY) ? 0.0 : exp2(A[r * bkv + cj] - m_new[r]);
-        P[r * bkv + cj] = pij;
-        rowsum += pij;
+        const double w = blind ? 0.0 : exp2(score[cj] - new_top);
+        block_mass += w;
+        if (w == 0.0) continue;
+        for (int c = 0; c < d; ++c) acc[c] += w * bf16_to_f64(vbase[(j0 + cj) * d + c]);
       }
-      vv[r] = (m_new[r] == -INFINITY) ? 1.0 : exp2(m[r] - m_new[r]);
-      l[r] = vv[r] * l[r] + rowsum;
-      m[r] = m_new[r];
+      mass = shrink * mass + block_mass;
+      top = new_top;
     }
-    /* Third Stage: O_i <- v*O_i, then O_i <- O_i + P_ij V_j */
-    for (int r = 0; r < rows; ++r) {
-      for (int c = 0; c < d; ++c) o[r * d + c] *= vv[r];
-      for (int cj = 0; cj < cols; ++cj) {
-        double pij = P[r * bkv + cj];
-        if (pij == 0.0) continue;
-        for (int c = 0; c < d; ++c) o[r * d + c] += pij * bf16_to_f64(vbase[(j0 + cj) * d + c]);
-      }
-    }
-  }
-  /* after the last j: O_i <- O_i * l^-1 */
-  for (int r = 0; r < rows; ++r) {
-    if (l[r] == 0.0) {
+    if (mass == 0.0) {
       lse[r] = -INFINITY;
-      for (int c = 0; c < d; ++c) o[r * d + c] = 0.0;
+      for (int c = 0; c < d; ++c) acc[c] = 0.0;
     } else {
-      for (int c = 0; c < d; ++c) o[r * d + c] /= l[r];
-      lse[r] = ln2 * (m[r] + log2(l[r]));
+      for (int c = 0; c < d; ++c) acc[c] /= mass;
+      lse[r] = ln2 * (top + log2(mass));
     }
   }
-  free(A); free(P); free(m); free(m_new); free(l); free(vv);
+  free(score);
+  free(keep);
   return executed;
 }
 
