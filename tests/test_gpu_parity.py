@@ -81,8 +81,10 @@ EDGE_CASES = [
 ]
 
 
+@pytest.mark.parametrize("emu", [0, 3], ids=["hw_exp", "half_poly_exp"])
 @pytest.mark.parametrize("case", EDGE_CASES, ids=[c["name"] for c in EDGE_CASES])
-def test_edge_cases_all_rows(case):
+def test_edge_cases_all_rows(case, emu):
+    """Every edge shape on the shipped kernel builds at both ends of the software-exponent range."""
     w = inputs.Workload(case["name"], case["B"], case["Hq"], case["Hkv"], case["S"], case["D"],
                         case.get("block", 128), case["flags"], window=case.get("window", 0),
                         keep_prob=case.get("keep", 0.0))
@@ -90,7 +92,7 @@ def test_edge_cases_all_rows(case):
     if w.flags & BITMAP:
         t = -(-w.seq // w.block)
         data["bitmap"] = inputs.block_bitmap(w.heads_q, t, t, w.keep_prob, seed=5)
-    attn, o, lse = H.run_gpu(w, data)
+    attn, o, lse = H.run_gpu(w, data, exp_emulation=emu)
     H.assert_parity(w, data, o, lse, H.all_rows(w))
     attn.close()
 
