@@ -66,8 +66,8 @@ struct Ctrl {
   long long timeout_cycles;
 };
 
-// Command word (producer -> MMA issuer): one word carries PV(s, t), S(s, t + 1) or both (the usual
-// case: the second product of a step is followed at once by the first product of the next step).
+// Command word (producer -> MMA issuer): one word carries S(s, t + 1), PV(s, t) or both (the usual
+// case: the first product of the next step is issued right before the second product of this one).
 constexpr uint32_t kCmdValid = 1u << 0, kCmdHasPV = 1u << 1, kCmdHasS = 1u << 2, kCmdSlot1 = 1u << 3,
                    kCmdVRingShift = 4, kCmdKRingShift = 8,  // 4 bits each: ring slot of the V / K tile
                    kCmdVPhase = 1u << 12, kCmdKPhase = 1u << 13, kCmdVSkipWait = 1u << 14, kCmdKSkipWait = 1u << 15,
@@ -157,8 +157,9 @@ __device__ __forceinline__ uint2 load_step(const Item &w, const StepPair *steps,
 // For each step t: first S(s, t) of slots that start at t, then for each present slot S(s, t + 1)
 // followed by PV(s, t): the first product runs one step ahead of the second, so a slot's next scores
 // are computed while its softmax warps still work on the current ones (they hold them in registers;
-// the S buffer in TMEM is free again as soon as they are loaded).  A tile wanted by both slots in one step is one ring fill: slot 0 uses
-// it first, slot 1 last (the planner guarantees lo0 <= lo1).  `ring` counts fills.
+// the S buffer in TMEM is free again as soon as they are loaded).  A tile wanted by both slots in
+// one step is one ring fill: slot 0 uses it first, slot 1 last (the planner guarantees lo0 <= lo1).
+// `ring` counts fills.
 // op(s, t, j, is_s, fill, first, last) returns false to stop.
 struct RingPos {
   uint32_t slot, phase;  // next fill goes to `slot`; `phase` flips each time the ring wraps
@@ -408,6 +409,7 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
 #endif
   uint32_t cmd = fifo_pop_warp(ctrl, head, p.status, lane);
   while (!(cmd & kCmdExit)) {
+    // look at the next command now, so that its shared-memory latency hides behind this one's issue
     volatile uint32_t *next_cell = &ctrl.fifo[head];
     __syncwarp();
     const uint32_t next_raw = *next_cell;
@@ -416,8 +418,12 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
     const bool has_pv = (cmd & kCmdHasPV) != 0, has_s = (cmd & kCmdHasS) != 0;
     constexpr uint32_t kRare = kCmdWaitOEmpty | kCmdWaitQFull | kCmdOEnd | kCmdQEnd;
     const uint32_t rare = cmd & kRare;
+    // One elected lane does the barrier work and issues; the other lanes only keep the loop's
+    // control values uniform.
     if (elect_one()) {
       TRACE_T0();
+      // test the barriers the command depends on back to back, so their latencies overlap; only
+      // the ones not yet complete are then waited for
       const bool need_v = has_pv && !(cmd & kCmdVSkipWait), need_k = has_s && !(cmd & kCmdKSkipWait);
       const bool need_f = has_s && (cmd & kCmdWaitSFree);
       uint64_t *s_free = &ctrl.s_free;
@@ -425,11 +431,20 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
       bool ok_k = !need_k || mbar_test_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u);
       bool ok_v = !need_v || mbar_test_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u);
       if (has_s) {
+        // S(s, t + 1) into the shared S buffer: its previous content must be in its owners' registers
         if (rare | uint32_t(!ok_f) | uint32_t(!ok_k)) {
           if (cmd & kCmdWaitQFull)
             ok = bounded_wait(&ctrl.q_full[s], (cmd & kCmdQFullPhase) ? 1u : 0u, ctrl, p.status);
-          if (ok && !ok_f) { TRACE_T0(); ok = bounded_wait(s_free, (cmd & kCmdSFreePhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(0); }
-          if (ok && !ok_k) { TRACE_T0(); ok = bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(1); }
+          if (ok && !ok_f) {
+            TRACE_T0();
+            ok = bounded_wait(s_free, (cmd & kCmdSFreePhase) ? 1u : 0u, ctrl, p.status);
+            TRACE_ADD(0);
+          }
+          if (ok && !ok_k) {
+            TRACE_T0();
+            ok = bounded_wait(&ctrl.ring_full[k_slot], (cmd & kCmdKPhase) ? 1u : 0u, ctrl, p.status);
+            TRACE_ADD(1);
+          }
         }
         if (ok) {
           tc_fence_after();
@@ -446,12 +461,21 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
         }
       }
       if (ok && has_pv) {
+        // O_s += P_s V: P from its own TMEM columns, written by the softmax warps of slot s
         const uint32_t p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
         const bool ok_p = mbar_test_wait(&ctrl.p_full[s], p_phase);
         if (rare | uint32_t(!ok_p) | uint32_t(!ok_v)) {
           if (cmd & kCmdWaitOEmpty) ok = bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status);
-          if (ok && !ok_v) { TRACE_T0(); ok = bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status); TRACE_ADD(2); }
-          if (ok && !ok_p) { TRACE_T0(); ok = bounded_wait(&ctrl.p_full[s], p_phase, ctrl, p.status); TRACE_ADD(3); }
+          if (ok && !ok_v) {
+            TRACE_T0();
+            ok = bounded_wait(&ctrl.ring_full[v_slot], (cmd & kCmdVPhase) ? 1u : 0u, ctrl, p.status);
+            TRACE_ADD(2);
+          }
+          if (ok && !ok_p) {
+            TRACE_T0();
+            ok = bounded_wait(&ctrl.p_full[s], p_phase, ctrl, p.status);
+            TRACE_ADD(3);
+          }
         }
         if (ok) {
           tc_fence_after();
