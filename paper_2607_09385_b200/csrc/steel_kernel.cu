@@ -455,15 +455,19 @@ __device__ void mma_role(const KernelParams &p, Ctrl &ctrl, uint8_t *smem_q, uin
             const uint64_t off = uint64_t(((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4);
             mma_ss(tmem + C::kColS, dq + off, dk + off, idesc_s, kk > 0);
           }
-          tc_commit(&ctrl.s_full[s]);
-          tc_commit_if(&ctrl.ring_empty[k_slot], cmd & kCmdKFinal);
-          if (rare) tc_commit_if(&ctrl.q_empty[s], cmd & kCmdQEnd);
         }
+      }
+      // A commit does not return before the instructions it covers have nearly drained, so the
+      // test of the next group's barrier goes between issuing this group and committing it.
+      const uint32_t p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
+      const bool ok_p = !has_pv || mbar_test_wait(&ctrl.p_full[s], p_phase);
+      if (ok && has_s) {
+        tc_commit(&ctrl.s_full[s]);
+        tc_commit_if(&ctrl.ring_empty[k_slot], cmd & kCmdKFinal);
+        if (rare) tc_commit_if(&ctrl.q_empty[s], cmd & kCmdQEnd);
       }
       if (ok && has_pv) {
         // O_s += P_s V: P from its own TMEM columns, written by the softmax warps of slot s
-        const uint32_t p_phase = (cmd & kCmdPPhase) ? 1u : 0u;
-        const bool ok_p = mbar_test_wait(&ctrl.p_full[s], p_phase);
         if (rare | uint32_t(!ok_p) | uint32_t(!ok_v)) {
           if (cmd & kCmdWaitOEmpty) ok = bounded_wait(&ctrl.o_empty[s], (cmd & kCmdOEmptyPhase) ? 1u : 0u, ctrl, p.status);
           if (ok && !ok_v) {
