@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0  # vendor figure for dense bf16 on one B200 (contex
 # from the ncu capture summarised in profiles/ (None until a capture exists for a workload).
 NCU_TRAFFIC_BYTES = {"c2_causal_s4k_mha32": 100930304 + 11335936,          # one-pass captures of one full launch each
                      "c3_window4k_s16k_gqa32x8": 213756928 + 99447296,
-                     "c4_bitmap25_s32k_h16": 408786176 + 118737408,
+                     "c4_bitmap25_s32k_h16": 413043200 + 119604736,
                      "c5_causal_s128k_gqa32x8": 3695049472 + 1193544192}
 
 
