@@ -34,8 +34,12 @@
 namespace steel {
 
 constexpr int kThreads = 384;        // softmax slot 0, softmax slot 1, {producer, MMA, 2 idle warps}
-constexpr int kRegsSoftmax = 216;    // registers per thread after the warpgroups re-split the file
+// Registers per thread after the warpgroups re-split the file.  2 * 128 * kRegsSoftmax + 128 *
+// kRegsOther must stay below the 65 536 registers of an SM with room to spare: setmaxnreg.inc waits,
+// without any bound, until the increase can be granted.
+constexpr int kRegsSoftmax = 216;
 constexpr int kRegsOther = 72;
+static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 65536 - 1024, "register re-split needs slack");
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;           // lazy rescale: P stays below 2^8
